@@ -1,0 +1,174 @@
+/*
+ * zellige.h -- C ABI of the coalesced attention engine for NVIDIA B200 (sm_100a).
+ *
+ * The engine executes, on one GPU, what the paper's Section IV-D ("Coalesced Attention
+ * Engine") assigns to one rank: every whole sequence placed on the rank (packed
+ * block-diagonally, never attending across sequences) together with the rank's shards of
+ * distributed-attention groups, in ONE launch.  A shard task is one query chunk attending
+ * to one K/V chunk; it produces a partial output plus a log-sum-exp, and partial results
+ * of the same query chunk are combined by a log-sum-exp merge (exact attention under
+ * context parallelism, Sections II-B and IV-A).  The K/V chunks that context parallelism
+ * would exchange between ranks are plain local inputs here.
+ *
+ * Conventions
+ *   - Two packed token spaces.  Q-space holds Q, O, dO, dQ and LSE (total_q rows);
+ *     KV-space holds K, V, dK, dV (total_kv rows).  Whole sequence i owns rows
+ *     [cu_seqlens[i], cu_seqlens[i+1]) of BOTH spaces.  Shard chunks are addressed by the
+ *     offsets in their descriptor and must lie at or after cu_seqlens[n_whole].
+ *   - Tensors are [tokens, n_heads, head_dim], contiguous, bf16, base 16-byte aligned.
+ *     LSE is [n_heads, total_q] fp32: natural log of the sum of exp(scale * q.k).
+ *   - Attention is bidirectional: no mask, bias or dropout.  head_dim is 64 or 128.
+ *   - All tensor arguments are DEVICE pointers unless marked host.  The caller owns every
+ *     tensor, the workspace and the stream; the library allocates only the small tables
+ *     inside a zl_tasks handle.
+ *   - Every function returns a zl_status; nothing throws, aborts or traps.  Kernels bound
+ *     all their waits; a wait that expires records ZL_ERR_TIMEOUT in the handle's device
+ *     status word (zl_last_device_status) and the kernel returns normally.
+ *   - Outputs land at the input token offsets whatever the internal work order
+ *     (Section IV-D: outputs keep the rank-local input order).
+ *   - A handle may be in flight on one stream at a time.
+ */
+#ifndef ZELLIGE_H_
+#define ZELLIGE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ZL_OK = 0,
+    ZL_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer, bad ordering of cu_seqlens */
+    ZL_ERR_OVERLAP = 2,     /* ranges that partially overlap, duplicates, a shard inside the whole region */
+    ZL_ERR_UNSUPPORTED = 3, /* head_dim not in {64,128}, or a device that is not sm_100 */
+    ZL_ERR_WORKSPACE = 4,   /* workspace smaller than zl_tasks_info.bwd_workspace_bytes */
+    ZL_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed */
+    ZL_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by zl_last_device_status) */
+} zl_status;
+
+/* One shard task: query rows [q_off, q_off+q_len) of Q-space attend to key rows
+ * [kv_off, kv_off+kv_len) of KV-space.  seq_id labels the long sequence the chunks belong
+ * to; tasks that share a query range must share seq_id.  Units: tokens. */
+typedef struct {
+    int32_t q_off, q_len, kv_off, kv_len, seq_id;
+} zl_shard_desc;
+
+typedef struct zl_tasks zl_tasks; /* opaque, immutable after zl_build_tasks */
+
+typedef struct {
+    int32_t n_tasks;        /* whole sequences + shard tasks with q_len > 0 */
+    int32_t n_merge_groups; /* distinct shard query ranges */
+    int32_t n_kv_groups;    /* distinct key ranges (backward work units) */
+    int32_t n_fwd_items;    /* forward work items (task, head, query block) */
+    int32_t n_bwd_items;    /* backward work items (kv group, head, key tile) */
+    int64_t partial_rows;   /* rows of o_partial / columns of lse_partial (slots are padded) */
+    size_t o_partial_bytes;     /* partial_rows * n_heads * head_dim * 4 */
+    size_t lse_partial_bytes;   /* n_heads * partial_rows * 4 */
+    size_t bwd_workspace_bytes; /* scratch needed by zl_coalesced_attn_bwd */
+} zl_tasks_info;
+
+/* zl_build_tasks -- lower a placement into the rank-local schedule (Section IV-D: "lowers
+ * the placement into a rank-local schedule and coalesces compatible segments").
+ *
+ *   cu_seqlens  host, n_whole+1 entries, cu[0]=0, non-decreasing; may be NULL if n_whole=0.
+ *   shards      host, n_shards descriptors; may be NULL if n_shards=0.
+ *   total_q/kv  rows of the two token spaces.
+ *   stream      cudaStream_t (as void*) used for the one small table upload.
+ *   out         receives the handle; free with zl_free_tasks.
+ *
+ * Every whole sequence becomes a task whose result is final after the forward launch.
+ * Every shard becomes a task that writes a partial result into a slot of o_partial /
+ * lse_partial.  Shard tasks with identical (q_off, q_len) form a merge group; tasks with
+ * identical (kv_off, kv_len) form a kv group whose dK/dV contributions are summed.  Work
+ * lists are ordered longest-first (by key length, then rows in the block; ties by task,
+ * head, block) so that a long video cannot straggle the launch.
+ *
+ * Validation (host only): any two query ranges must be identical or disjoint, likewise
+ * key ranges (ZL_ERR_OVERLAP); shard ranges lie inside the totals and at or after
+ * cu_seqlens[n_whole]; within a merge group key ranges are pairwise disjoint and seq_id
+ * agrees; duplicate (query range, key range) pairs are rejected.  Zero-length whole
+ * sequences and shards with q_len = 0 are accepted and ignored; a shard with kv_len = 0
+ * contributes an empty partial (O = 0, LSE = -inf). */
+zl_status zl_build_tasks(const int32_t* cu_seqlens, int32_t n_whole,
+                         const zl_shard_desc* shards, int32_t n_shards,
+                         int32_t total_q, int32_t total_kv, int32_t n_heads, int32_t head_dim,
+                         void* stream, zl_tasks** out);
+
+zl_status zl_tasks_get_info(const zl_tasks* tasks, zl_tasks_info* info);
+
+/* Slot of shard `shard_idx` (index into the `shards` array given to zl_build_tasks) inside
+ * o_partial / lse_partial: rows [row_off, row_off + q_len) hold the task's partial result,
+ * rows_padded >= q_len is the slot size.  Shards with q_len = 0 report rows_padded = 0. */
+zl_status zl_tasks_get_partial_slot(const zl_tasks* tasks, int32_t shard_idx,
+                                    int64_t* row_off, int64_t* rows_padded);
+
+/* Host copies of the work lists, for inspection and tests.  Each forward item is 4 int32:
+ * (task, head, first query row of the block relative to the task, rows in the block); each
+ * backward item is 4 int32: (kv group, head, first key row relative to the group, rows).
+ * `items` may be NULL to query the count only. */
+zl_status zl_tasks_get_fwd_items(const zl_tasks* tasks, int32_t* items, int32_t capacity, int32_t* count);
+zl_status zl_tasks_get_bwd_items(const zl_tasks* tasks, int32_t* items, int32_t capacity, int32_t* count);
+
+void zl_free_tasks(zl_tasks* tasks);
+
+/* zl_coalesced_attn_fwd -- one persistent launch over the whole work list (Section IV-D:
+ * whole sequences packed into one block-diagonal attention call, shards run beside them).
+ *
+ *   q            [total_q, H, d] bf16        k, v  [total_kv, H, d] bf16
+ *   scale        multiplies q.k before the softmax (1/sqrt(d) in every named workload)
+ *   o            [total_q, H, d] bf16; rows of whole sequences are final on return of the
+ *                launch, rows of shard query ranges are untouched until zl_lse_merge
+ *   lse          [H, total_q] fp32, same rule
+ *   o_partial    [partial_rows, H, d] fp32: per shard task softmax(S_t) V_t, i.e.
+ *                normalised within the task's own K/V chunk (unnormalised with respect to
+ *                the union of chunks); may be NULL when there are no shards
+ *   lse_partial  [H, partial_rows] fp32: per shard task log-sum-exp over its chunk
+ *
+ * Asynchronous on `stream`.  Scores between tokens of different tasks are never formed;
+ * masked tail scores are selected to -inf, never multiplied.  Inputs must be finite. */
+zl_status zl_coalesced_attn_fwd(const zl_tasks* tasks, const void* q, const void* k, const void* v,
+                                float scale, void* o, float* lse,
+                                float* o_partial, float* lse_partial, void* stream);
+
+/* zl_lse_merge -- combine the partial results of every merge group (the accumulation step
+ * of ring / all-gather context parallelism, Section II-B):
+ *     LSE = log sum_t exp(LSE_t),   O = sum_t exp(LSE_t - LSE) * O_t
+ * summed in ascending shard order (bit-deterministic).  Writes final bf16 O and fp32 LSE at
+ * the group's query rows.  Rows whose parts are all empty get O = 0, LSE = -inf. */
+zl_status zl_lse_merge(const zl_tasks* tasks, const float* o_partial, const float* lse_partial,
+                       void* o, float* lse, void* stream);
+
+/* zl_coalesced_attn_bwd -- gradients of every task in one call, for dL/dO = d_o and no
+ * gradient through LSE.  With P = exp(scale*QK^T - LSE) recomputed from the FINAL
+ * (merged) LSE and D_i = sum_c dO_ic O_ic from the FINAL O:
+ *     dV = P^T dO,  dS = P o (dO V^T - D),  dQ = scale * dS K,  dK = scale * dS^T Q.
+ * dQ is summed over tasks sharing a query range, dK/dV over tasks sharing a key range
+ * (on a context-parallel rank that is the contribution of the local queries only).
+ *
+ *   o, lse       final forward results;  d_o [total_q, H, d] bf16
+ *   dq           [total_q, H, d] bf16;   dk, dv [total_kv, H, d] bf16.  Rows covered by at
+ *                least one task are overwritten; rows covered by none are left untouched.
+ *   workspace    device scratch of at least zl_tasks_info.bwd_workspace_bytes, 256-byte
+ *                aligned; contents need not be initialised and are clobbered.
+ * Asynchronous on `stream` (three launches: preprocess, main, dQ conversion). */
+zl_status zl_coalesced_attn_bwd(const zl_tasks* tasks, const void* q, const void* k, const void* v,
+                                const void* o, const float* lse, const void* d_o, float scale,
+                                void* dq, void* dk, void* dv,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises the handle's device and reads the device status word written by the
+ * kernels: code is ZL_OK or ZL_ERR_TIMEOUT, `where` identifies the wait that expired
+ * (kernel id * 1000 + site).  Resets the word to ZL_OK. */
+zl_status zl_last_device_status(const zl_tasks* tasks, int32_t* code, int32_t* where);
+
+const char* zl_status_str(zl_status s);
+
+/* Number of this library's kernel launches enqueued since load (all handles). */
+int64_t zl_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZELLIGE_H_ */

@@ -1,0 +1,198 @@
+"""ctypes binding of libzellige.so -- same names as the C ABI in include/zellige.h.
+
+Argument marshalling only.  Tensors are torch CUDA tensors (device memory and streams come
+from PyTorch); the functions pass their data pointers and the current stream to the
+library.  Raw-pointer entry points (``*_ptr``) take integers so that callers holding host
+buffers can drive the same C calls.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libzellige.so")
+
+STATUS_NAMES = {0: "ZL_OK", 1: "ZL_ERR_INVALID_ARG", 2: "ZL_ERR_OVERLAP", 3: "ZL_ERR_UNSUPPORTED",
+                4: "ZL_ERR_WORKSPACE", 5: "ZL_ERR_CUDA", 6: "ZL_ERR_TIMEOUT"}
+
+
+class ZlError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {STATUS_NAMES.get(status, status)}")
+
+
+class ShardDesc(ctypes.Structure):
+    _fields_ = [("q_off", ctypes.c_int32), ("q_len", ctypes.c_int32), ("kv_off", ctypes.c_int32),
+                ("kv_len", ctypes.c_int32), ("seq_id", ctypes.c_int32)]
+
+
+class TasksInfo(ctypes.Structure):
+    _fields_ = [("n_tasks", ctypes.c_int32), ("n_merge_groups", ctypes.c_int32),
+                ("n_kv_groups", ctypes.c_int32), ("n_fwd_items", ctypes.c_int32),
+                ("n_bwd_items", ctypes.c_int32), ("partial_rows", ctypes.c_int64),
+                ("o_partial_bytes", ctypes.c_size_t), ("lse_partial_bytes", ctypes.c_size_t),
+                ("bwd_workspace_bytes", ctypes.c_size_t)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2608_01150_b200.build` "
+            "(nvcc, sm_100a). There is no fallback path.")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64)
+    lib.zl_build_tasks.restype = ctypes.c_int
+    lib.zl_build_tasks.argtypes = [vp, i32, vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+    lib.zl_tasks_get_info.restype = ctypes.c_int
+    lib.zl_tasks_get_info.argtypes = [vp, ctypes.POINTER(TasksInfo)]
+    lib.zl_tasks_get_partial_slot.restype = ctypes.c_int
+    lib.zl_tasks_get_partial_slot.argtypes = [vp, i32, i64p, i64p]
+    for name in ("zl_tasks_get_fwd_items", "zl_tasks_get_bwd_items"):
+        getattr(lib, name).restype = ctypes.c_int
+        getattr(lib, name).argtypes = [vp, vp, i32, ctypes.POINTER(i32)]
+    lib.zl_free_tasks.restype = None
+    lib.zl_free_tasks.argtypes = [vp]
+    lib.zl_coalesced_attn_fwd.restype = ctypes.c_int
+    lib.zl_coalesced_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
+    lib.zl_lse_merge.restype = ctypes.c_int
+    lib.zl_lse_merge.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.zl_coalesced_attn_bwd.restype = ctypes.c_int
+    lib.zl_coalesced_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp,
+                                          ctypes.c_size_t, vp]
+    lib.zl_last_device_status.restype = ctypes.c_int
+    lib.zl_last_device_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.zl_status_str.restype = ctypes.c_char_p
+    lib.zl_status_str.argtypes = [ctypes.c_int]
+    lib.zl_launch_count.restype = ctypes.c_int64
+    lib.zl_launch_count.argtypes = []
+    return lib
+
+
+_lib = _load()
+
+
+def lib():
+    return _lib
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise ZlError(status, what)
+
+
+def _stream_ptr(stream=None) -> int:
+    import torch
+    if stream is None:
+        if not torch.cuda.is_available():
+            return 0
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+class TaskHandle:
+    """Owns a ``zl_tasks*``.  Built once per placement, reused for every layer and step."""
+
+    def __init__(self, ptr: int, n_heads: int, head_dim: int, total_q: int, total_kv: int, n_shards: int):
+        self._ptr = ctypes.c_void_p(ptr)
+        self.n_heads, self.head_dim, self.total_q, self.total_kv = n_heads, head_dim, total_q, total_kv
+        self.n_shards = n_shards
+        info = TasksInfo()
+        _check(_lib.zl_tasks_get_info(self._ptr, ctypes.byref(info)), "zl_tasks_get_info")
+        self.info = info
+
+    @property
+    def ptr(self):
+        return self._ptr
+
+    def partial_slot(self, shard_idx: int) -> Tuple[int, int]:
+        a, b = ctypes.c_int64(), ctypes.c_int64()
+        _check(_lib.zl_tasks_get_partial_slot(self._ptr, shard_idx, ctypes.byref(a), ctypes.byref(b)),
+               "zl_tasks_get_partial_slot")
+        return a.value, b.value
+
+    def _items(self, fn) -> List[Tuple[int, int, int, int]]:
+        n = ctypes.c_int32()
+        _check(fn(self._ptr, None, 0, ctypes.byref(n)), "items count")
+        buf = (ctypes.c_int32 * (4 * max(1, n.value)))()
+        _check(fn(self._ptr, buf, n.value, ctypes.byref(n)), "items")
+        return [tuple(buf[4 * i:4 * i + 4]) for i in range(n.value)]
+
+    def fwd_items(self):
+        return self._items(_lib.zl_tasks_get_fwd_items)
+
+    def bwd_items(self):
+        return self._items(_lib.zl_tasks_get_bwd_items)
+
+    def last_device_status(self) -> Tuple[int, int]:
+        c, w = ctypes.c_int32(), ctypes.c_int32()
+        _check(_lib.zl_last_device_status(self._ptr, ctypes.byref(c), ctypes.byref(w)), "zl_last_device_status")
+        return c.value, w.value
+
+    def close(self):
+        if self._ptr:
+            _lib.zl_free_tasks(self._ptr)
+            self._ptr = ctypes.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def build_tasks(cu_seqlens: Sequence[int], shards: Sequence[Sequence[int]], total_q: int, total_kv: int,
+                n_heads: int, head_dim: int, stream=None) -> TaskHandle:
+    """zl_build_tasks: placement (cu_seqlens + shard descriptors) -> task handle."""
+    n_whole = max(0, len(cu_seqlens) - 1)
+    cu = (ctypes.c_int32 * max(1, len(cu_seqlens)))(*[int(c) for c in cu_seqlens])
+    sh = (ShardDesc * max(1, len(shards)))(*[ShardDesc(*[int(v) for v in s]) for s in shards])
+    out = ctypes.c_void_p()
+    st = _lib.zl_build_tasks(ctypes.cast(cu, ctypes.c_void_p) if len(cu_seqlens) else None, n_whole,
+                             ctypes.cast(sh, ctypes.c_void_p) if len(shards) else None, len(shards),
+                             total_q, total_kv, n_heads, head_dim, _stream_ptr(stream), ctypes.byref(out))
+    _check(st, "zl_build_tasks")
+    return TaskHandle(out.value, n_heads, head_dim, total_q, total_kv, len(shards))
+
+
+def coalesced_attn_fwd(tasks: TaskHandle, q, k, v, scale: float, o, lse, o_partial=None, lse_partial=None,
+                       stream=None):
+    """zl_coalesced_attn_fwd.  Tensors: torch CUDA tensors or raw device pointers (int)."""
+    _check(_lib.zl_coalesced_attn_fwd(tasks.ptr, _ptr(q), _ptr(k), _ptr(v), ctypes.c_float(scale), _ptr(o),
+                                      _ptr(lse), _ptr(o_partial), _ptr(lse_partial), _stream_ptr(stream)),
+           "zl_coalesced_attn_fwd")
+
+
+def lse_merge(tasks: TaskHandle, o_partial, lse_partial, o, lse, stream=None):
+    """zl_lse_merge."""
+    _check(_lib.zl_lse_merge(tasks.ptr, _ptr(o_partial), _ptr(lse_partial), _ptr(o), _ptr(lse),
+                             _stream_ptr(stream)), "zl_lse_merge")
+
+
+def coalesced_attn_bwd(tasks: TaskHandle, q, k, v, o, lse, d_o, scale: float, dq, dk, dv, workspace,
+                       workspace_bytes: Optional[int] = None, stream=None):
+    """zl_coalesced_attn_bwd."""
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(_lib.zl_coalesced_attn_bwd(tasks.ptr, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o),
+                                      ctypes.c_float(scale), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
+                                      ctypes.c_size_t(workspace_bytes), _stream_ptr(stream)),
+           "zl_coalesced_attn_bwd")
+
+
+def launch_count() -> int:
+    return int(_lib.zl_launch_count())

@@ -1,0 +1,301 @@
+// C-ABI layer of libzellige: handle management, TMA descriptor encoding, kernel launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "zl_device.h"
+
+namespace zl {
+cudaError_t launch_bwd(int head_dim, const struct BwdLaunch& b, cudaStream_t stream);
+}
+
+using namespace zl;
+
+struct zl_tasks {
+    Schedule sched;
+    int device = -1;           // -1: host-only handle (no CUDA device present)
+    int n_sms = 0;
+    uint8_t* d_tables = nullptr;  // one allocation holding every device table
+    Task* d_tasks = nullptr;
+    WorkItem* d_fwd_items = nullptr;
+    WorkItem* d_bwd_items = nullptr;
+    MergeGroup* d_merge_groups = nullptr;
+    int32_t* d_merge_parts = nullptr;
+    int32_t* d_merge_prefix = nullptr;
+    KvGroup* d_kv_groups = nullptr;
+    int32_t* d_kv_group_tasks = nullptr;
+    int32_t* d_status = nullptr;
+};
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Tensor map over a packed [rows, H, d] bf16 tensor: box = 64 columns x 1 head x box_rows rows,
+// 128-byte swizzle, zero fill outside the tensor.
+bool make_tmap(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim, int box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)(rows > 0 ? rows : 1)};
+    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)head_dim * 2 * n_heads};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+template <class T>
+size_t place(size_t& off, size_t count) {
+    off = align_up(off, 256);
+    const size_t at = off;
+    off += count * sizeof(T);
+    return at;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* zl_status_str(zl_status s) {
+    switch (s) {
+        case ZL_OK: return "ZL_OK";
+        case ZL_ERR_INVALID_ARG: return "ZL_ERR_INVALID_ARG";
+        case ZL_ERR_OVERLAP: return "ZL_ERR_OVERLAP";
+        case ZL_ERR_UNSUPPORTED: return "ZL_ERR_UNSUPPORTED";
+        case ZL_ERR_WORKSPACE: return "ZL_ERR_WORKSPACE";
+        case ZL_ERR_CUDA: return "ZL_ERR_CUDA";
+        case ZL_ERR_TIMEOUT: return "ZL_ERR_TIMEOUT";
+    }
+    return "ZL_ERR_UNKNOWN";
+}
+
+int64_t zl_launch_count(void) { return g_launches.load(); }
+
+zl_status zl_build_tasks(const int32_t* cu_seqlens, int32_t n_whole, const zl_shard_desc* shards,
+                         int32_t n_shards, int32_t total_q, int32_t total_kv, int32_t n_heads,
+                         int32_t head_dim, void* stream, zl_tasks** out) {
+    if (!out) return ZL_ERR_INVALID_ARG;
+    *out = nullptr;
+    zl_tasks* h = new (std::nothrow) zl_tasks();
+    if (!h) return ZL_ERR_INVALID_ARG;
+    zl_status st = build_schedule(cu_seqlens, n_whole, shards, n_shards, total_q, total_kv, n_heads, head_dim,
+                                  &h->sched);
+    if (st != ZL_OK) { delete h; return st; }
+
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) {
+        cudaGetLastError();  // host-only handle: inspection works, launches return ZL_ERR_CUDA
+        *out = h;
+        return ZL_OK;
+    }
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        delete h; return ZL_ERR_CUDA;
+    }
+    if (prop.major != 10) { delete h; return ZL_ERR_UNSUPPORTED; }
+    h->device = dev;
+    h->n_sms = prop.multiProcessorCount;
+
+    const Schedule& s = h->sched;
+    size_t off = 0;
+    const size_t o_tasks = place<Task>(off, s.tasks.size());
+    const size_t o_fwd = place<WorkItem>(off, s.fwd_items.size());
+    const size_t o_bwd = place<WorkItem>(off, s.bwd_items.size());
+    const size_t o_mg = place<MergeGroup>(off, s.merge_groups.size());
+    const size_t o_mp = place<int32_t>(off, s.merge_parts.size());
+    const size_t o_mr = place<int32_t>(off, s.merge_row_prefix.size());
+    const size_t o_kg = place<KvGroup>(off, s.kv_groups.size());
+    const size_t o_kt = place<int32_t>(off, s.kv_group_tasks.size());
+    const size_t o_st = place<int32_t>(off, 2);
+    const size_t total = align_up(off, 256);
+
+    std::vector<uint8_t> host(total, 0);
+    auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host.data() + at, src, bytes); };
+    put(o_tasks, s.tasks.data(), s.tasks.size() * sizeof(Task));
+    put(o_fwd, s.fwd_items.data(), s.fwd_items.size() * sizeof(WorkItem));
+    put(o_bwd, s.bwd_items.data(), s.bwd_items.size() * sizeof(WorkItem));
+    put(o_mg, s.merge_groups.data(), s.merge_groups.size() * sizeof(MergeGroup));
+    put(o_mp, s.merge_parts.data(), s.merge_parts.size() * sizeof(int32_t));
+    put(o_mr, s.merge_row_prefix.data(), s.merge_row_prefix.size() * sizeof(int32_t));
+    put(o_kg, s.kv_groups.data(), s.kv_groups.size() * sizeof(KvGroup));
+    put(o_kt, s.kv_group_tasks.data(), s.kv_group_tasks.size() * sizeof(int32_t));
+
+    if (cudaMalloc(&h->d_tables, total) != cudaSuccess) { delete h; return ZL_ERR_CUDA; }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    // pageable source: the copy is staged before the call returns, so `host` may go away
+    if (cudaMemcpyAsync(h->d_tables, host.data(), total, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaStreamSynchronize(cs) != cudaSuccess) {
+        cudaFree(h->d_tables); delete h; return ZL_ERR_CUDA;
+    }
+    h->d_tasks = reinterpret_cast<Task*>(h->d_tables + o_tasks);
+    h->d_fwd_items = reinterpret_cast<WorkItem*>(h->d_tables + o_fwd);
+    h->d_bwd_items = reinterpret_cast<WorkItem*>(h->d_tables + o_bwd);
+    h->d_merge_groups = reinterpret_cast<MergeGroup*>(h->d_tables + o_mg);
+    h->d_merge_parts = reinterpret_cast<int32_t*>(h->d_tables + o_mp);
+    h->d_merge_prefix = reinterpret_cast<int32_t*>(h->d_tables + o_mr);
+    h->d_kv_groups = reinterpret_cast<KvGroup*>(h->d_tables + o_kg);
+    h->d_kv_group_tasks = reinterpret_cast<int32_t*>(h->d_tables + o_kt);
+    h->d_status = reinterpret_cast<int32_t*>(h->d_tables + o_st);
+    *out = h;
+    return ZL_OK;
+}
+
+zl_status zl_tasks_get_info(const zl_tasks* t, zl_tasks_info* info) {
+    if (!t || !info) return ZL_ERR_INVALID_ARG;
+    const Schedule& s = t->sched;
+    info->n_tasks = (int32_t)s.tasks.size();
+    info->n_merge_groups = (int32_t)s.merge_groups.size();
+    info->n_kv_groups = (int32_t)s.kv_groups.size();
+    info->n_fwd_items = (int32_t)s.fwd_items.size();
+    info->n_bwd_items = (int32_t)s.bwd_items.size();
+    info->partial_rows = s.partial_rows;
+    info->o_partial_bytes = (size_t)s.partial_rows * s.n_heads * s.head_dim * sizeof(float);
+    info->lse_partial_bytes = (size_t)s.partial_rows * s.n_heads * sizeof(float);
+    info->bwd_workspace_bytes = s.bwd_workspace_bytes;
+    return ZL_OK;
+}
+
+zl_status zl_tasks_get_partial_slot(const zl_tasks* t, int32_t shard_idx, int64_t* row_off, int64_t* rows_padded) {
+    if (!t || !row_off || !rows_padded) return ZL_ERR_INVALID_ARG;
+    if (shard_idx < 0 || shard_idx >= (int32_t)t->sched.shard_to_task.size()) return ZL_ERR_INVALID_ARG;
+    *row_off = t->sched.shard_slot_off[shard_idx];
+    *rows_padded = t->sched.shard_slot_rows[shard_idx];
+    return ZL_OK;
+}
+
+static zl_status copy_items(const std::vector<WorkItem>& v, int32_t* items, int32_t capacity, int32_t* count) {
+    if (!count) return ZL_ERR_INVALID_ARG;
+    *count = (int32_t)v.size();
+    if (!items) return ZL_OK;
+    if (capacity < (int32_t)v.size()) return ZL_ERR_INVALID_ARG;
+    if (!v.empty()) std::memcpy(items, v.data(), v.size() * sizeof(WorkItem));
+    return ZL_OK;
+}
+
+zl_status zl_tasks_get_fwd_items(const zl_tasks* t, int32_t* items, int32_t capacity, int32_t* count) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    return copy_items(t->sched.fwd_items, items, capacity, count);
+}
+
+zl_status zl_tasks_get_bwd_items(const zl_tasks* t, int32_t* items, int32_t capacity, int32_t* count) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    return copy_items(t->sched.bwd_items, items, capacity, count);
+}
+
+void zl_free_tasks(zl_tasks* t) {
+    if (!t) return;
+    if (t->d_tables) cudaFree(t->d_tables);
+    delete t;
+}
+
+zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k, const void* v, float scale,
+                                void* o, float* lse, float* o_partial, float* lse_partial, void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    const Schedule& s = t->sched;
+    if (s.fwd_items.empty()) return ZL_OK;
+    if (t->device < 0) return ZL_ERR_CUDA;
+    if (!q || !k || !v || !o || !lse) return ZL_ERR_INVALID_ARG;
+    if (s.partial_rows > 0 && (!o_partial || !lse_partial)) return ZL_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(o_partial))
+        return ZL_ERR_INVALID_ARG;
+    if (!(scale > 0.f) || !std::isfinite(scale)) return ZL_ERR_INVALID_ARG;
+
+    CUtensorMap tq, tk, tv;
+    if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ) ||
+        !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
+        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV))
+        return ZL_ERR_CUDA;
+
+    FwdParams p{};
+    p.tasks = t->d_tasks;
+    p.items = t->d_fwd_items;
+    p.n_items = (int32_t)s.fwd_items.size();
+    p.n_heads = s.n_heads;
+    p.total_q = s.total_q;
+    p.partial_rows = (int32_t)s.partial_rows;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
+    p.o_partial = o_partial;
+    p.lse_partial = lse_partial;
+    p.status = t->d_status;
+    const int grid = std::min<int>(t->n_sms, p.n_items);
+    if (launch_fwd(s.head_dim, tq, tk, tv, p, grid, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return ZL_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return ZL_OK;
+}
+
+zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* lse_partial, void* o, float* lse,
+                       void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    const Schedule& s = t->sched;
+    if (s.merge_groups.empty()) return ZL_OK;
+    if (t->device < 0) return ZL_ERR_CUDA;
+    if (!o_partial || !lse_partial || !o || !lse) return ZL_ERR_INVALID_ARG;
+    if (!aligned16(o_partial) || !aligned16(o)) return ZL_ERR_INVALID_ARG;
+    MergeParams p{};
+    p.groups = t->d_merge_groups;
+    p.parts = t->d_merge_parts;
+    p.row_prefix = t->d_merge_prefix;
+    p.n_groups = (int32_t)s.merge_groups.size();
+    p.n_heads = s.n_heads;
+    p.total_q = s.total_q;
+    p.partial_rows = (int32_t)s.partial_rows;
+    p.o_partial = o_partial;
+    p.lse_partial = lse_partial;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
+    if (launch_merge(s.head_dim, p, t->n_sms, static_cast<cudaStream_t>(stream)) != cudaSuccess) return ZL_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return ZL_OK;
+}
+
+zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k, const void* v, const void* o,
+                                const float* lse, const void* d_o, float scale, void* dq, void* dk, void* dv,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    (void)t; (void)q; (void)k; (void)v; (void)o; (void)lse; (void)d_o; (void)scale; (void)dq; (void)dk; (void)dv;
+    (void)workspace; (void)workspace_bytes; (void)stream;
+    return ZL_ERR_UNSUPPORTED;
+}
+
+zl_status zl_last_device_status(const zl_tasks* t, int32_t* code, int32_t* where) {
+    if (!t || !code || !where) return ZL_ERR_INVALID_ARG;
+    *code = ZL_OK; *where = 0;
+    if (t->device < 0) return ZL_OK;
+    int32_t host[2] = {0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) return ZL_ERR_CUDA;
+    if (cudaMemcpy(host, t->d_status, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return ZL_ERR_CUDA;
+    *code = host[0]; *where = host[1];
+    if (host[0] != 0 && cudaMemset(t->d_status, 0, sizeof(host)) != cudaSuccess) return ZL_ERR_CUDA;
+    return ZL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,45 @@
+// Kernel parameter blocks and launch entry points shared by the C-ABI layer and the kernels.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "zl_internal.h"
+
+namespace zl {
+
+struct FwdParams {
+    const Task* tasks;
+    const WorkItem* items;
+    int32_t n_items;
+    int32_t n_heads;
+    int32_t total_q;
+    int32_t partial_rows;
+    float scale_log2;  // scale * log2(e)
+    __nv_bfloat16* o;
+    float* lse;
+    float* o_partial;
+    float* lse_partial;
+    int32_t* status;  // [0] = code, [1] = where
+};
+
+struct MergeParams {
+    const MergeGroup* groups;
+    const int32_t* parts;       // partial slot row offsets
+    const int32_t* row_prefix;  // n_groups + 1
+    int32_t n_groups;
+    int32_t n_heads;
+    int32_t total_q;
+    int32_t partial_rows;
+    const float* o_partial;
+    const float* lse_partial;
+    __nv_bfloat16* o;
+    float* lse;
+};
+
+cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                       const FwdParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_merge(int head_dim, const MergeParams& p, int n_sms, cudaStream_t stream);
+
+}  // namespace zl

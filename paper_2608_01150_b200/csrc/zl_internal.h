@@ -1,0 +1,66 @@
+// Internal definitions shared by the host scheduler and the kernels of libzellige.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "zellige.h"
+
+namespace zl {
+
+constexpr int kTileQ = 128;   // query rows per MMA tile (TMEM lanes)
+constexpr int kTileKV = 128;  // key rows per MMA tile
+constexpr int kFwdBlockQ = kTileQ;  // query rows per forward work item
+
+// One attention task on the device: whole sequence or shard.
+struct alignas(32) Task {
+    int32_t q_off, q_len, kv_off, kv_len;
+    int32_t partial_slot;  // first row of the task's slot in o_partial, -1 for a whole sequence
+    int32_t merge_group;   // -1 for a whole sequence
+    int32_t kv_group;
+    int32_t q_group;       // index of the distinct query range (dQ accumulation unit)
+};
+
+// (task | kv group, head, first row relative to the task's query range | group's key range, rows)
+struct alignas(16) WorkItem {
+    int32_t unit, head, row0, rows;
+};
+
+struct alignas(16) MergeGroup {
+    int32_t q_off, q_len;
+    int32_t part_begin, n_parts;  // range in the merge part list (partial slot row offsets)
+};
+
+struct alignas(16) KvGroup {
+    int32_t kv_off, kv_len;
+    int32_t task_begin, n_tasks;  // range in the kv-group task list
+};
+
+// Everything zl_build_tasks derives from a placement, on the host.
+struct Schedule {
+    int32_t n_heads = 0, head_dim = 0, total_q = 0, total_kv = 0;
+    std::vector<Task> tasks;
+    std::vector<int32_t> shard_to_task;     // per input shard: task index or -1 (q_len == 0)
+    std::vector<int32_t> shard_slot_off;    // per input shard: slot row offset (or 0)
+    std::vector<int32_t> shard_slot_rows;   // per input shard: padded slot rows (0 if skipped)
+    std::vector<MergeGroup> merge_groups;
+    std::vector<int32_t> merge_parts;       // slot row offsets, ascending shard order per group
+    std::vector<int32_t> merge_row_prefix;  // n_merge_groups+1 prefix sums of q_len
+    std::vector<KvGroup> kv_groups;
+    std::vector<int32_t> kv_group_tasks;
+    std::vector<WorkItem> fwd_items;
+    std::vector<WorkItem> bwd_items;
+    int64_t partial_rows = 0;
+    size_t bwd_workspace_bytes = 0;
+    // byte offsets inside the backward workspace
+    size_t ws_dq_acc_off = 0, ws_delta_off = 0;
+};
+
+// Validates the placement and fills `s`.  Pure host code, no CUDA.
+zl_status build_schedule(const int32_t* cu_seqlens, int32_t n_whole, const zl_shard_desc* shards,
+                         int32_t n_shards, int32_t total_q, int32_t total_kv, int32_t n_heads,
+                         int32_t head_dim, Schedule* s);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace zl

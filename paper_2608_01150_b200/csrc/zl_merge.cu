@@ -1,0 +1,93 @@
+// LSE merge kernel: combines the partial results of the shard tasks of each merge group
+// (the accumulation step of ring / all-gather context parallelism, paper Section II-B):
+//     LSE = M + log sum_t exp(LSE_t - M),  M = max_t LSE_t
+//     O   = sum_t exp(LSE_t - LSE) * O_t        (ascending shard order, bit-deterministic)
+// HBM-bound: one warp per (query row, head), each lane owns head_dim/32 consecutive floats
+// and reads them with one vector load per part.
+#include <cuda_runtime.h>
+
+#include "zl_device.h"
+
+namespace zl {
+
+namespace {
+
+constexpr int kMergeThreads = 256;
+
+template <int D>
+__global__ void __launch_bounds__(kMergeThreads) zl_merge_kernel(const MergeParams p) {
+    constexpr int V = D / 32;  // floats per lane: 4 (d=128) or 2 (d=64)
+    const int lane = threadIdx.x & 31;
+    const int warps_per_block = kMergeThreads / 32;
+    const int64_t n_rows = p.row_prefix[p.n_groups];
+    const int64_t n_units = n_rows * p.n_heads;
+    for (int64_t u = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); u < n_units;
+         u += (int64_t)gridDim.x * warps_per_block) {
+        const int64_t r = u / p.n_heads;
+        const int h = (int)(u - r * p.n_heads);
+        // group of flat row r: binary search over the prefix sums
+        int lo = 0, hi = p.n_groups;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (p.row_prefix[mid] <= r) lo = mid; else hi = mid;
+        }
+        const MergeGroup g = p.groups[lo];
+        const int row = (int)(r - p.row_prefix[lo]);
+        float M = -INFINITY;
+        for (int t = 0; t < g.n_parts; ++t) {
+            const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
+            M = fmaxf(M, __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr));
+        }
+        float z = 0.f;
+        for (int t = 0; t < g.n_parts; ++t) {
+            const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
+            const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
+            z += (M == -INFINITY) ? 0.f : expf(lt - M);
+        }
+        const float L = (M == -INFINITY) ? -INFINITY : M + logf(z);
+        float acc[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc[i] = 0.f;
+        for (int t = 0; t < g.n_parts; ++t) {
+            const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
+            const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
+            const float w = (L == -INFINITY) ? 0.f : expf(lt - L);
+            const float* src = p.o_partial + (pr * p.n_heads + h) * D + lane * V;
+            if constexpr (V == 4) {
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
+                acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+                acc[2] = fmaf(w, x.z, acc[2]); acc[3] = fmaf(w, x.w, acc[3]);
+            } else {
+                const float2 x = __ldcs(reinterpret_cast<const float2*>(src));
+                acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+            }
+        }
+        const int64_t qrow = (int64_t)g.q_off + row;
+        __nv_bfloat16* dst = p.o + (qrow * p.n_heads + h) * D + lane * V;
+        if constexpr (V == 4) {
+            __nv_bfloat162 a = __floats2bfloat162_rn(acc[0], acc[1]);
+            __nv_bfloat162 b = __floats2bfloat162_rn(acc[2], acc[3]);
+            uint2 o2;
+            o2.x = *reinterpret_cast<uint32_t*>(&a);
+            o2.y = *reinterpret_cast<uint32_t*>(&b);
+            *reinterpret_cast<uint2*>(dst) = o2;
+        } else {
+            *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(acc[0], acc[1]);
+        }
+        if (lane == 0) p.lse[(int64_t)h * p.total_q + qrow] = L;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_merge(int head_dim, const MergeParams& p, int n_sms, cudaStream_t stream) {
+    if (p.n_groups == 0) return cudaSuccess;
+    const int grid = n_sms * 8;  // 8 resident blocks of 256 threads per SM
+    if (head_dim == 128)
+        zl_merge_kernel<128><<<grid, kMergeThreads, 0, stream>>>(p);
+    else
+        zl_merge_kernel<64><<<grid, kMergeThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace zl

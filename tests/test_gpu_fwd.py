@@ -1,0 +1,137 @@
+"""GPU parity of the forward path (zl_coalesced_attn_fwd + zl_lse_merge) against the fp64
+CPU oracle, called through the C ABI via the Python binding."""
+import numpy as np
+import pytest
+import torch
+
+import zl_workloads as W
+from oracle import attention as A
+from zl_testlib import (GpuRun, bits, check_forward, dev_to_f64, random_bits, to_dev, to_f64,
+                        GATE_O_MAX, GATE_LSE_MAX, SENTINEL)
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(p, Qb, Kb, Vb, gate=True):
+    run = GpuRun(p)
+    O, LSE, OP, LP = run.forward(to_dev(Qb), to_dev(Kb), to_dev(Vb))
+    ref = A.placement_fwd(p, to_f64(Qb), to_f64(Kb), to_f64(Vb))
+    stats = check_forward(p, O, LSE, ref)
+    if gate:
+        assert stats["o_excess"] <= GATE_O_MAX and stats["lse_max"] <= GATE_LSE_MAX, stats
+    return run, (O, LSE, OP, LP), ref, stats
+
+
+def test_config1_forward_and_partials():
+    p = W.config(1)
+    Qb, Kb, Vb = bits(p, "Q"), bits(p, "K"), bits(p, "V")
+    run, (O, LSE, OP, LP), ref, stats = _run(p, Qb, Kb, Vb)
+    # per-task partials: normalised within their own K/V chunk
+    OPh, LPh = dev_to_f64(OP), dev_to_f64(LP)
+    for si, s in enumerate(p.shards):
+        off, padded = run.h.partial_slot(si)
+        assert padded == 1024
+        o_t, l_t = ref["partials"][si]
+        assert np.abs(OPh[off:off + s[1]] - o_t).max() <= GATE_O_MAX
+        assert np.abs(LPh[:, off:off + s[1]] - l_t).max() <= GATE_LSE_MAX
+
+
+EDGE = [1, 2, 15, 16, 17, 127, 128, 129, 255, 256, 257]
+
+
+@pytest.mark.parametrize("d,H", [(64, 1), (128, 3)])
+def test_tile_edge_lengths_whole(d, H):
+    """Whole sequences whose lengths straddle every tile edge, packed in one launch."""
+    p = W.make_placement("edges", H, d, 11, EDGE + [24 + 128, 16 + 256, 126, 106 + 128, 6, 104])
+    rng = np.random.RandomState(d + H)
+    Qb, Kb, Vb = (random_bits(rng, p.total_q, H, d) for _ in range(3))
+    _run(p, Qb, Kb, Vb)
+
+
+@pytest.mark.parametrize("lq,lkv", [(1, 1), (1, 257), (257, 1), (129, 127), (17, 255), (130, 300)])
+def test_tile_edge_lengths_shards(lq, lkv):
+    d, H = 128, 2
+    p = W.custom_placement("edge_shard", H, d, 5, [0, 40], [(40, lq, 40, lkv, 0), (40, lq, 40 + lkv, 3, 0)],
+                           40 + lq + 5, 40 + lkv + 3 + 7)
+    rng = np.random.RandomState(lq * 1000 + lkv)
+    Qb = random_bits(rng, p.total_q, H, d)
+    Kb = random_bits(rng, p.total_kv, H, d)
+    Vb = random_bits(rng, p.total_kv, H, d)
+    _run(p, Qb, Kb, Vb)
+
+
+def test_spike_keys_at_tile_and_chunk_boundaries():
+    """A key aligned with a query makes that query's output equal that key's value row, so
+    a dropped, duplicated or leaked key is an O(1) error."""
+    d, H = 128, 1
+    p = W.make_placement("spike", H, d, 3, [300, 200], [(1, 2, 260)])
+    rng = np.random.RandomState(9)
+    Q = rng.standard_normal((p.total_q, H, d)).astype(np.float32)
+    K = rng.standard_normal((p.total_kv, H, d)).astype(np.float32) * 0.1
+    V = rng.standard_normal((p.total_kv, H, d)).astype(np.float32)
+    beta = 4.0
+    # (query row, key row) pairs inside the same logical problem
+    pairs = [(0, 0), (5, 127), (6, 128), (7, 255), (8, 256), (9, 299),          # whole seq 0 (300)
+             (300, 300), (301, 499),                                             # whole seq 1 (200)
+             (500, 500), (501, 627), (502, 628), (503, 759), (504, 760), (505, 1019)]  # shard chunks
+    for qi, kj in pairs:
+        K[kj] = beta * Q[qi]
+    # spikes in NEIGHBOURING problems must have no effect
+    K[300 - 1] = K[300 - 1]  # (last key of seq 0 is already a spike target of row 9)
+    Qb, Kb, Vb = (W.f32_to_bf16_bits(W._bf16_round_f32(x)) for x in (Q, K, V))
+    run, (O, LSE, OP, LP), ref, stats = _run(p, Qb, Kb, Vb, gate=False)
+    Og = dev_to_f64(O)
+    Vf = to_f64(Vb)
+    for qi, kj in pairs:
+        assert np.abs(ref["O"][qi, 0] - Vf[kj, 0]).max() < 1e-6, "spike too weak for the test"
+        assert np.abs(Og[qi, 0] - Vf[kj, 0]).max() < 2e-2, (qi, kj)
+
+
+def test_isolation_and_untouched_rows():
+    """Perturbing one sequence leaves every other sequence's output bit-identical, and rows
+    that belong to no task keep their previous contents."""
+    d, H = 64, 2
+    p = W.custom_placement("iso", H, d, 1, [0, 100, 230], [(240, 50, 240, 70, 0)], 300, 320)
+    rng = np.random.RandomState(2)
+    Qb, Kb, Vb = random_bits(rng, 300, H, d), random_bits(rng, 320, H, d), random_bits(rng, 320, H, d)
+    run, (O1, L1, _, _), ref, _ = _run(p, Qb, Kb, Vb)
+    Q2, K2, V2 = Qb.copy(), Kb.copy(), Vb.copy()
+    big = W.f32_to_bf16_bits(np.full((1,), 3e38, dtype=np.float32))[0]
+    K2[100:230] = big                     # large finite poison in sequence 1
+    V2[100:230] = big
+    K2[230:240] = big                     # and in rows no task owns
+    run2 = GpuRun(p)
+    O2, L2, _, _ = run2.forward(to_dev(Q2), to_dev(K2), to_dev(V2))
+    keep = np.r_[0:100, 240:290]
+    assert torch.equal(O1[keep], O2[keep]) and torch.equal(L1[:, keep], L2[:, keep])
+    assert torch.all(O2[290:] == SENTINEL) and torch.all(O2[230:240] == SENTINEL)
+
+
+def test_forward_is_run_to_run_bit_identical():
+    p = W.config(1)
+    Qd, Kd, Vd = to_dev(bits(p, "Q")), to_dev(bits(p, "K")), to_dev(bits(p, "V"))
+    run = GpuRun(p)
+    a = run.forward(Qd, Kd, Vd)
+    b = run.forward(Qd, Kd, Vd)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_empty_kv_shard_and_single_part_group():
+    d, H = 64, 1
+    p = W.custom_placement("empty", H, d, 1, [0, 10], [(10, 20, 10, 0, 0), (30, 5, 10, 33, 1)], 40, 50)
+    rng = np.random.RandomState(4)
+    Qb, Kb, Vb = random_bits(rng, 40, H, d), random_bits(rng, 50, H, d), random_bits(rng, 50, H, d)
+    run, (O, LSE, _, _), ref, _ = _run(p, Qb, Kb, Vb)
+    assert torch.all(O[10:30] == 0) and torch.all(torch.isneginf(LSE[:, 10:30]))
+
+
+def test_randomised_small_placements():
+    rng = np.random.RandomState(1234)
+    for trial in range(6):
+        d = int(rng.choice([64, 128]))
+        H = int(rng.randint(1, 4))
+        p = W.random_placement(rng, H, d)
+        Qb = random_bits(rng, p.total_q, H, d)
+        Kb = random_bits(rng, p.total_kv, H, d)
+        Vb = random_bits(rng, p.total_kv, H, d)
+        _run(p, Qb, Kb, Vb)
