@@ -9,10 +9,6 @@
 
 #include "zl_device.h"
 
-namespace zl {
-cudaError_t launch_bwd(int head_dim, const struct BwdLaunch& b, cudaStream_t stream);
-}
-
 using namespace zl;
 
 struct zl_tasks {
@@ -26,6 +22,7 @@ struct zl_tasks {
     MergeGroup* d_merge_groups = nullptr;
     int32_t* d_merge_parts = nullptr;
     int32_t* d_merge_prefix = nullptr;
+    QGroup* d_q_groups = nullptr;
     KvGroup* d_kv_groups = nullptr;
     int32_t* d_kv_group_tasks = nullptr;
     int32_t* d_status = nullptr;
@@ -131,6 +128,7 @@ zl_status zl_build_tasks(const int32_t* cu_seqlens, int32_t n_whole, const zl_sh
     const size_t o_mg = place<MergeGroup>(off, s.merge_groups.size());
     const size_t o_mp = place<int32_t>(off, s.merge_parts.size());
     const size_t o_mr = place<int32_t>(off, s.merge_row_prefix.size());
+    const size_t o_qg = place<QGroup>(off, s.q_groups.size());
     const size_t o_kg = place<KvGroup>(off, s.kv_groups.size());
     const size_t o_kt = place<int32_t>(off, s.kv_group_tasks.size());
     const size_t o_st = place<int32_t>(off, 2);
@@ -144,6 +142,7 @@ zl_status zl_build_tasks(const int32_t* cu_seqlens, int32_t n_whole, const zl_sh
     put(o_mg, s.merge_groups.data(), s.merge_groups.size() * sizeof(MergeGroup));
     put(o_mp, s.merge_parts.data(), s.merge_parts.size() * sizeof(int32_t));
     put(o_mr, s.merge_row_prefix.data(), s.merge_row_prefix.size() * sizeof(int32_t));
+    put(o_qg, s.q_groups.data(), s.q_groups.size() * sizeof(QGroup));
     put(o_kg, s.kv_groups.data(), s.kv_groups.size() * sizeof(KvGroup));
     put(o_kt, s.kv_group_tasks.data(), s.kv_group_tasks.size() * sizeof(int32_t));
 
@@ -160,6 +159,7 @@ zl_status zl_build_tasks(const int32_t* cu_seqlens, int32_t n_whole, const zl_sh
     h->d_merge_groups = reinterpret_cast<MergeGroup*>(h->d_tables + o_mg);
     h->d_merge_parts = reinterpret_cast<int32_t*>(h->d_tables + o_mp);
     h->d_merge_prefix = reinterpret_cast<int32_t*>(h->d_tables + o_mr);
+    h->d_q_groups = reinterpret_cast<QGroup*>(h->d_tables + o_qg);
     h->d_kv_groups = reinterpret_cast<KvGroup*>(h->d_tables + o_kg);
     h->d_kv_group_tasks = reinterpret_cast<int32_t*>(h->d_tables + o_kt);
     h->d_status = reinterpret_cast<int32_t*>(h->d_tables + o_st);
@@ -281,9 +281,62 @@ zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* l
 zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k, const void* v, const void* o,
                                 const float* lse, const void* d_o, float scale, void* dq, void* dk, void* dv,
                                 void* workspace, size_t workspace_bytes, void* stream) {
-    (void)t; (void)q; (void)k; (void)v; (void)o; (void)lse; (void)d_o; (void)scale; (void)dq; (void)dk; (void)dv;
-    (void)workspace; (void)workspace_bytes; (void)stream;
-    return ZL_ERR_UNSUPPORTED;
+    if (!t) return ZL_ERR_INVALID_ARG;
+    const Schedule& s = t->sched;
+    if (s.tasks.empty()) return ZL_OK;
+    if (t->device < 0) return ZL_ERR_CUDA;
+    if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !workspace) return ZL_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv) || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
+        return ZL_ERR_INVALID_ARG;
+    if (!(scale > 0.f) || !std::isfinite(scale)) return ZL_ERR_INVALID_ARG;
+    if (workspace_bytes < s.bwd_workspace_bytes) return ZL_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+    CUtensorMap tq, tk, tv, tdo;
+    if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ) ||
+        !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
+        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
+        !make_tmap(&tdo, d_o, s.total_q, s.n_heads, s.head_dim, kTileQ))
+        return ZL_ERR_CUDA;
+
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    BwdParams p{};
+    p.tasks = t->d_tasks;
+    p.items = t->d_bwd_items;
+    p.kv_groups = t->d_kv_groups;
+    p.kv_group_tasks = t->d_kv_group_tasks;
+    p.q_groups = t->d_q_groups;
+    p.n_items = (int32_t)s.bwd_items.size();
+    p.n_q_groups = (int32_t)s.q_groups.size();
+    p.n_heads = s.n_heads;
+    p.total_q = s.total_q;
+    p.q_pad_total = (int32_t)s.q_pad_total;
+    p.scale = scale;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.o = static_cast<const __nv_bfloat16*>(o);
+    p.d_o = static_cast<const __nv_bfloat16*>(d_o);
+    p.lse = lse;
+    p.dq = static_cast<__nv_bfloat16*>(dq);
+    p.dk = static_cast<__nv_bfloat16*>(dk);
+    p.dv = static_cast<__nv_bfloat16*>(dv);
+    p.dq_acc = reinterpret_cast<float*>(ws + s.ws_dq_acc_off);
+    p.lse2 = reinterpret_cast<float*>(ws + s.ws_lse2_off);
+    p.delta = reinterpret_cast<float*>(ws + s.ws_delta_off);
+    p.status = t->d_status;
+
+    if (cudaMemsetAsync(p.dq_acc, 0, (size_t)s.q_pad_total * s.n_heads * s.head_dim * sizeof(float), cs) != cudaSuccess)
+        return ZL_ERR_CUDA;
+    if (launch_bwd_pre(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+    g_launches.fetch_add(1);
+    if (p.n_items > 0) {
+        const int grid = std::min<int>(t->n_sms, p.n_items);
+        if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
+        g_launches.fetch_add(1);
+    }
+    if (launch_bwd_post(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return ZL_OK;
 }
 
 zl_status zl_last_device_status(const zl_tasks* t, int32_t* code, int32_t* where) {

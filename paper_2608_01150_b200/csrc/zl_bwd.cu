@@ -1,0 +1,484 @@
+// Backward kernels of the coalesced attention engine (sm_100a).
+//
+// Gradients of softmax attention for every task of a placement (whole sequences and
+// context-parallel shard tasks, paper Section IV-D), for dL/dO = dO and no gradient
+// through LSE.  With P = exp(scale * Q K^T - LSE) recomputed from the final LSE:
+//     dV = P^T dO,   dS = P o (dO V^T - D),   dQ = scale * dS K,   dK = scale * dS^T Q,
+//     D_i = sum_c dO_ic O_ic.
+//
+// Three launches:
+//   pre   D and LSE*log2(e) into padded per-query-range scratch rows (the dQ accumulator is
+//         cleared by a memset node before it);
+//   main  persistent; a CTA owns one 128-row key tile of one kv group and one head, keeps
+//         K, V in shared memory and dK, dV in TMEM, and loops over every 128-row query tile
+//         of every task that shares the key range.  Per tile it issues five tcgen05 MMAs
+//         (S^T = K Q^T, dP^T = V dO^T, dV += P^T dO, dK += dS^T Q, dQ = dS K); dK/dV need no
+//         atomics, dQ tiles are added into an fp32 accumulator with vector reductions;
+//   post  dQ accumulator * scale -> bf16.
+#include <cuda_runtime.h>
+
+#include "zl_device.h"
+#include "zl_ptx.cuh"
+
+namespace zl {
+
+using namespace ptx;
+
+namespace {
+
+constexpr uint64_t kWaitLimitNs = 4000000000ull;
+
+// ======================================================================= preprocess
+constexpr int kPreThreads = 256;
+
+__device__ __forceinline__ int find_q_group(const QGroup* g, int n, int slot_row) {
+    int lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (g[mid].slot <= slot_row) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kPreThreads) zl_bwd_pre_kernel(const BwdParams p) {
+    constexpr int V = D / 32;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_units = (int64_t)p.q_pad_total * p.n_heads;
+    for (int64_t u = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); u < n_units;
+         u += (int64_t)gridDim.x * (kPreThreads / 32)) {
+        const int slot_row = (int)(u / p.n_heads);
+        const int h = (int)(u - (int64_t)slot_row * p.n_heads);
+        const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, slot_row)];
+        const int r = slot_row - g.slot;
+        float delta = 0.f, l2 = INFINITY;
+        if (r < g.q_len) {
+            const int64_t row = (int64_t)g.q_off + r;
+            const __nv_bfloat16* po = p.o + (row * p.n_heads + h) * D + lane * V;
+            const __nv_bfloat16* pd = p.d_o + (row * p.n_heads + h) * D + lane * V;
+            float acc = 0.f;
+#pragma unroll
+            for (int i = 0; i < V; i += 2) {
+                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + i));
+                const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pd + i));
+                acc = fmaf(a.x, b.x, acc);
+                acc = fmaf(a.y, b.y, acc);
+            }
+#pragma unroll
+            for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+            delta = acc;
+            const float l = p.lse[(int64_t)h * p.total_q + row];
+            l2 = (l == -INFINITY) ? INFINITY : l * 1.4426950408889634f;
+        }
+        if (lane == 0) {
+            p.delta[(int64_t)h * p.q_pad_total + slot_row] = delta;
+            p.lse2[(int64_t)h * p.q_pad_total + slot_row] = l2;
+        }
+    }
+}
+
+// ======================================================================= post
+template <int D>
+__global__ void __launch_bounds__(kPreThreads) zl_bwd_post_kernel(const BwdParams p) {
+    constexpr int V = D / 32;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_units = (int64_t)p.q_pad_total * p.n_heads;
+    for (int64_t u = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); u < n_units;
+         u += (int64_t)gridDim.x * (kPreThreads / 32)) {
+        const int slot_row = (int)(u / p.n_heads);
+        const int h = (int)(u - (int64_t)slot_row * p.n_heads);
+        const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, slot_row)];
+        const int r = slot_row - g.slot;
+        if (r >= g.q_len) continue;
+        const float* src = p.dq_acc + ((int64_t)slot_row * p.n_heads + h) * D + lane * V;
+        __nv_bfloat16* dst = p.dq + (((int64_t)g.q_off + r) * p.n_heads + h) * D + lane * V;
+        if constexpr (V == 4) {
+            const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
+            uint2 o2;
+            o2.x = pack_bf16(x.x * p.scale, x.y * p.scale);
+            o2.y = pack_bf16(x.z * p.scale, x.w * p.scale);
+            *reinterpret_cast<uint2*>(dst) = o2;
+        } else {
+            const float2 x = __ldcs(reinterpret_cast<const float2*>(src));
+            *reinterpret_cast<uint32_t*>(dst) = pack_bf16(x.x * p.scale, x.y * p.scale);
+        }
+    }
+}
+
+// ======================================================================= main
+constexpr int kBwdThreads = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 P/dS, warps 6-9 dQ
+
+template <int D>
+struct BwdSmem {
+    static constexpr int kStages = (D == 128) ? 1 : 2;
+    static constexpr int kTileBytes = 128 * D * 2;
+    static constexpr int kBoxBytes = 128 * 128;
+    static constexpr int kBoxes = D / 64;
+    alignas(1024) uint8_t k[kTileBytes];
+    alignas(1024) uint8_t v[kTileBytes];
+    alignas(1024) uint8_t q[kStages][kTileBytes];
+    alignas(1024) uint8_t d_o[kStages][kTileBytes];
+    alignas(1024) uint8_t ds[2 * kBoxBytes];  // dS^T tile: 128 key rows x 128 query columns, bf16
+    alignas(16) float lse2[kStages][128];
+    alignas(16) float delta[kStages][128];
+    alignas(8) uint64_t kv_full, kv_empty;
+    uint64_t qdo_full[kStages], qdo_empty[kStages];
+    uint64_t s_full, p_full, ds_full, dq_full, dq_empty, acc_full;
+    uint32_t tmem_base;
+    volatile int32_t abort_flag;
+};
+
+__device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_flag, int where) {
+    *abort_flag = 1;
+    if (atomicCAS(status, 0, (int)ZL_ERR_TIMEOUT) == 0) status[1] = where;
+}
+
+#define ZL_WAIT(bar, parity, site)                                        \
+    do {                                                                  \
+        if (!mbar_wait((bar), (parity), kWaitLimitNs) || sm.abort_flag) { \
+            report(p.status, &sm.abort_flag, 2000 + (site));              \
+            goto teardown;                                                \
+        }                                                                 \
+    } while (0)
+#define ZL_WAIT_WARP(bar, parity, site)                                              \
+    do {                                                                             \
+        const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs) && !sm.abort_flag; \
+        if (!__all_sync(0xffffffffu, ok_)) {                                         \
+            report(p.status, &sm.abort_flag, 2000 + (site));                         \
+            goto teardown;                                                           \
+        }                                                                            \
+    } while (0)
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                   const BwdParams p) {
+    using Smem = BwdSmem<D>;
+    constexpr int kStages = Smem::kStages;
+    constexpr int kBoxes = Smem::kBoxes;
+    extern __shared__ uint8_t smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    // TMEM columns: S^T / P^T [0,128), dP^T / dQ [128,256), dV [256,256+D), dK [384,384+D)
+    constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384, kTmemCols = 512;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sm.kv_full, 1);
+        mbar_init(&sm.kv_empty, 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sm.qdo_full[s], 1);
+            mbar_init(&sm.qdo_empty[s], 1);
+        }
+        mbar_init(&sm.s_full, 1);
+        mbar_init(&sm.p_full, 128);
+        mbar_init(&sm.ds_full, 128);
+        mbar_init(&sm.dq_full, 1);
+        mbar_init(&sm.dq_empty, 128);
+        mbar_init(&sm.acc_full, 1);
+        sm.abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tm_q);
+        prefetch_tmap(&tm_k);
+        prefetch_tmap(&tm_v);
+        prefetch_tmap(&tm_do);
+    }
+    if (warp == 1) {
+        tmem_alloc(&sm.tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t item_cnt = 0, it_cnt = 0;
+            for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
+                const WorkItem wi = p.items[it];
+                const KvGroup g = p.kv_groups[wi.unit];
+                ZL_WAIT(&sm.kv_empty, (item_cnt & 1) ^ 1, 1);
+                mbar_arrive_expect_tx(&sm.kv_full, 2 * Smem::kTileBytes);
+                for (int b = 0; b < kBoxes; ++b) {
+                    tma_load_3d(sm.k + b * Smem::kBoxBytes, &tm_k, &sm.kv_full, b * 64, wi.head, g.kv_off + wi.row0);
+                    tma_load_3d(sm.v + b * Smem::kBoxBytes, &tm_v, &sm.kv_full, b * 64, wi.head, g.kv_off + wi.row0);
+                }
+                for (int ti = 0; ti < g.n_tasks; ++ti) {
+                    const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
+                    const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
+                    for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
+                        const int s = it_cnt % kStages;
+                        ZL_WAIT(&sm.qdo_empty[s], ((it_cnt / kStages) & 1) ^ 1, 2);
+                        mbar_arrive_expect_tx(&sm.qdo_full[s], 2 * Smem::kTileBytes + 1024);
+                        for (int b = 0; b < kBoxes; ++b) {
+                            tma_load_3d(sm.q[s] + b * Smem::kBoxBytes, &tm_q, &sm.qdo_full[s], b * 64, wi.head,
+                                        t.q_off + qt * kTileQ);
+                            tma_load_3d(sm.d_o[s] + b * Smem::kBoxBytes, &tm_do, &sm.qdo_full[s], b * 64, wi.head,
+                                        t.q_off + qt * kTileQ);
+                        }
+                        const int64_t vec = (int64_t)wi.head * p.q_pad_total + t.q_slot + qt * kTileQ;
+                        bulk_load_1d(sm.lse2[s], p.lse2 + vec, 512, &sm.qdo_full[s]);
+                        bulk_load_1d(sm.delta[s], p.delta + vec, 512, &sm.qdo_full[s]);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: K-major x K-major
+            constexpr uint32_t idesc_dv = make_idesc_bf16(128, D, 0, 1);    // A in TMEM / K-major smem, B MN-major
+            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 1, 1);    // A MN-major smem, B MN-major
+            const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v), ds_addr = smem_u32(sm.ds);
+            uint32_t item_cnt = 0, it_cnt = 0;
+            for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
+                const WorkItem wi = p.items[it];
+                const KvGroup g = p.kv_groups[wi.unit];
+                ZL_WAIT(&sm.kv_full, item_cnt & 1, 11);
+                bool first = true;
+                for (int ti = 0; ti < g.n_tasks; ++ti) {
+                    const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
+                    const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
+                    for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
+                        const int s = it_cnt % kStages;
+                        const uint32_t q_addr = smem_u32(sm.q[s]), do_addr = smem_u32(sm.d_o[s]);
+                        ZL_WAIT(&sm.qdo_full[s], (it_cnt / kStages) & 1, 12);
+                        ZL_WAIT(&sm.dq_empty, (it_cnt & 1) ^ 1, 13);  // previous dQ tile drained
+                        tc_fence_after();
+#pragma unroll
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
+                            mma_ss(tmem + kColS, make_desc_sw128(k_addr + off, 16, 1024),
+                                   make_desc_sw128(q_addr + off, 16, 1024), idesc_s, ks > 0);
+                        }
+#pragma unroll
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
+                            mma_ss(tmem + kColDP, make_desc_sw128(v_addr + off, 16, 1024),
+                                   make_desc_sw128(do_addr + off, 16, 1024), idesc_s, ks > 0);
+                        }
+                        mma_commit(&sm.s_full);
+                        ZL_WAIT(&sm.p_full, it_cnt & 1, 14);
+                        tc_fence_after();
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
+                            mma_ts(tmem + kColDV, tmem + kColS + ks * 8,
+                                   make_desc_sw128(do_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv,
+                                   !first || ks > 0);
+                        ZL_WAIT(&sm.ds_full, it_cnt & 1, 15);
+                        tc_fence_after();
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
+                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
+                            mma_ss(tmem + kColDK, make_desc_sw128(ds_addr + off, 16, 1024),
+                                   make_desc_sw128(q_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv,
+                                   !first || ks > 0);
+                        }
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows
+                            mma_ss(tmem + kColDP, make_desc_sw128(ds_addr + ks * 2048, Smem::kBoxBytes, 1024),
+                                   make_desc_sw128(k_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dq, ks > 0);
+                        mma_commit(&sm.dq_full);
+                        mma_commit(&sm.qdo_empty[s]);
+                        first = false;
+                    }
+                }
+                mma_commit(&sm.acc_full);
+                mma_commit(&sm.kv_empty);
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------------ P / dS warps (one key row per thread)
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t ds_row_addr = smem_u32(sm.ds) + row * 128;
+        const float sl2 = p.scale_log2;
+        uint32_t item_cnt = 0, it_cnt = 0;
+        for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
+            const WorkItem wi = p.items[it];
+            const KvGroup g = p.kv_groups[wi.unit];
+            const bool row_ok = row < wi.rows;
+            for (int ti = 0; ti < g.n_tasks; ++ti) {
+                const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
+                const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
+                for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
+                    const int s = it_cnt % kStages;
+                    const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
+                    ZL_WAIT_WARP(&sm.qdo_full[s], (it_cnt / kStages) & 1, 21);  // lse2 / delta vectors
+                    ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 22);
+                    if (it_cnt > 0) ZL_WAIT_WARP(&sm.dq_full, (it_cnt - 1) & 1, 23);  // dS buffer consumed
+                    tc_fence_after();
+                    const bool full = row_ok && q_valid == kTileQ;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t sr[32], dr[32];
+                        tmem_ld_x32(lane_addr + kColS + c * 32, sr);
+                        tmem_ld_x32(lane_addr + kColDP + c * 32, dr);
+                        tmem_wait_ld();
+                        uint32_t pp[16], dd[16];
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            const int col = c * 32 + i;
+                            const float2 l2 = *reinterpret_cast<const float2*>(&sm.lse2[s][col]);
+                            const float2 dl = *reinterpret_cast<const float2*>(&sm.delta[s][col]);
+                            float p0 = ex2(fmaf(__uint_as_float(sr[i]), sl2, -l2.x));
+                            float p1 = ex2(fmaf(__uint_as_float(sr[i + 1]), sl2, -l2.y));
+                            float d0 = p0 * (__uint_as_float(dr[i]) - dl.x);
+                            float d1 = p1 * (__uint_as_float(dr[i + 1]) - dl.y);
+                            if (!full) {
+                                const bool ok0 = row_ok && col < q_valid, ok1 = row_ok && col + 1 < q_valid;
+                                p0 = ok0 ? p0 : 0.f; d0 = ok0 ? d0 : 0.f;
+                                p1 = ok1 ? p1 : 0.f; d1 = ok1 ? d1 : 0.f;
+                            }
+                            pp[i / 2] = pack_bf16(p0, p1);
+                            dd[i / 2] = pack_bf16(d0, d1);
+                        }
+                        tmem_st_x16(lane_addr + kColS + c * 16, pp);
+#pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            const int c16 = c * 4 + k4;  // 16-byte chunk index along the query axis
+                            const uint32_t addr = ds_row_addr + (c16 >> 3) * Smem::kBoxBytes + (((c16 & 7) ^ (row & 7)) << 4);
+                            st_shared_v4(addr, dd[k4 * 4], dd[k4 * 4 + 1], dd[k4 * 4 + 2], dd[k4 * 4 + 3]);
+                        }
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(&sm.p_full);
+                    fence_proxy_async_smem();
+                    mbar_arrive(&sm.ds_full);
+                }
+            }
+            // ---- epilogue: dV and dK of this key tile
+            ZL_WAIT_WARP(&sm.acc_full, item_cnt & 1, 24);
+            tc_fence_after();
+            const int64_t grow = (int64_t)g.kv_off + wi.row0 + row;
+            __nv_bfloat16* dv_dst = p.dv + (grow * p.n_heads + wi.head) * D;
+            __nv_bfloat16* dk_dst = p.dk + (grow * p.n_heads + wi.head) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_x32(lane_addr + kColDV + c * 32, r);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 o4;
+                        o4.x = pack_bf16(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                        o4.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                        o4.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+                        o4.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+                        *reinterpret_cast<uint4*>(dv_dst + c * 32 + i) = o4;
+                    }
+                }
+                tmem_ld_x32(lane_addr + kColDK + c * 32, r);
+                tmem_wait_ld();
+                if (row_ok) {
+                    const float sc = p.scale;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 o4;
+                        o4.x = pack_bf16(__uint_as_float(r[i]) * sc, __uint_as_float(r[i + 1]) * sc);
+                        o4.y = pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc);
+                        o4.z = pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc);
+                        o4.w = pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc);
+                        *reinterpret_cast<uint4*>(dk_dst + c * 32 + i) = o4;
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    } else {
+        // ------------------------------------------------------------------ dQ warps (one query row per thread)
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+        uint32_t it_cnt = 0;
+        for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
+            const WorkItem wi = p.items[it];
+            const KvGroup g = p.kv_groups[wi.unit];
+            for (int ti = 0; ti < g.n_tasks; ++ti) {
+                const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
+                const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
+                for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
+                    const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
+                    ZL_WAIT_WARP(&sm.dq_full, it_cnt & 1, 31);
+                    tc_fence_after();
+                    float* dst = p.dq_acc + (((int64_t)t.q_slot + qt * kTileQ + row) * p.n_heads + wi.head) * D;
+                    uint32_t r[D];
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t tmp[32];
+                        tmem_ld_x32(lane_addr + kColDP + c * 32, tmp);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[c * 32 + i] = tmp[i];
+                    }
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    mbar_arrive(&sm.dq_empty);
+                    if (row < q_valid) {
+#pragma unroll
+                        for (int i = 0; i < D; i += 4)
+                            red_add_v4(dst + i, __uint_as_float(r[i]), __uint_as_float(r[i + 1]),
+                                       __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                    }
+                }
+            }
+        }
+    }
+
+teardown:
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+template <int D>
+cudaError_t launch_main_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                          const CUtensorMap& tdo, const BwdParams& p, int grid, cudaStream_t stream) {
+    constexpr int smem = sizeof(BwdSmem<D>) + 1024;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(zl_bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    zl_bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream) {
+    if (p.q_pad_total == 0) return cudaSuccess;
+    const int grid = n_sms * 8;
+    if (head_dim == 128) zl_bwd_pre_kernel<128><<<grid, kPreThreads, 0, stream>>>(p);
+    else zl_bwd_pre_kernel<64><<<grid, kPreThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bwd_main(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                            const CUtensorMap& tdo, const BwdParams& p, int grid, cudaStream_t stream) {
+    if (p.n_items == 0) return cudaSuccess;
+    return head_dim == 128 ? launch_main_t<128>(tq, tk, tv, tdo, p, grid, stream)
+                           : launch_main_t<64>(tq, tk, tv, tdo, p, grid, stream);
+}
+
+cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream) {
+    if (p.q_pad_total == 0) return cudaSuccess;
+    const int grid = n_sms * 8;
+    if (head_dim == 128) zl_bwd_post_kernel<128><<<grid, kPreThreads, 0, stream>>>(p);
+    else zl_bwd_post_kernel<64><<<grid, kPreThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace zl

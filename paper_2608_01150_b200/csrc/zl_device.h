@@ -38,6 +38,36 @@ struct MergeParams {
     float* lse;
 };
 
+struct BwdParams {
+    const Task* tasks;
+    const WorkItem* items;       // (kv group, head, first key row, rows)
+    const KvGroup* kv_groups;
+    const int32_t* kv_group_tasks;
+    const QGroup* q_groups;
+    int32_t n_items;
+    int32_t n_q_groups;
+    int32_t n_heads;
+    int32_t total_q;
+    int32_t q_pad_total;
+    float scale;
+    float scale_log2;
+    const __nv_bfloat16* o;
+    const __nv_bfloat16* d_o;
+    const float* lse;
+    __nv_bfloat16* dq;
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    float* dq_acc;  // [q_pad_total, H, d]
+    float* lse2;    // [H, q_pad_total]: lse * log2(e), +inf on padding rows
+    float* delta;   // [H, q_pad_total]: rowsum(dO o O), 0 on padding rows
+    int32_t* status;
+};
+
+cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
+cudaError_t launch_bwd_main(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                            const CUtensorMap& tdo, const BwdParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
+
 cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                        const FwdParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_merge(int head_dim, const MergeParams& p, int n_sms, cudaStream_t stream);

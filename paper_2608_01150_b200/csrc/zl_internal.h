@@ -16,8 +16,8 @@ constexpr int kFwdBlockQ = kTileQ;  // query rows per forward work item
 struct alignas(32) Task {
     int32_t q_off, q_len, kv_off, kv_len;
     int32_t partial_slot;  // first row of the task's slot in o_partial, -1 for a whole sequence
-    int32_t merge_group;   // -1 for a whole sequence
-    int32_t kv_group;
+    int32_t q_slot;        // first row of the task's query range in the padded backward scratch
+    int32_t kv_group;      // -1 if kv_len == 0
     int32_t q_group;       // index of the distinct query range (dQ accumulation unit)
 };
 
@@ -29,6 +29,11 @@ struct alignas(16) WorkItem {
 struct alignas(16) MergeGroup {
     int32_t q_off, q_len;
     int32_t part_begin, n_parts;  // range in the merge part list (partial slot row offsets)
+};
+
+// A distinct query range: rows [slot, slot + pad128(q_len)) of the backward scratch arrays.
+struct alignas(16) QGroup {
+    int32_t q_off, q_len, slot, pad;
 };
 
 struct alignas(16) KvGroup {
@@ -46,6 +51,8 @@ struct Schedule {
     std::vector<MergeGroup> merge_groups;
     std::vector<int32_t> merge_parts;       // slot row offsets, ascending shard order per group
     std::vector<int32_t> merge_row_prefix;  // n_merge_groups+1 prefix sums of q_len
+    std::vector<QGroup> q_groups;
+    int64_t q_pad_total = 0;                // rows of the padded backward scratch arrays
     std::vector<KvGroup> kv_groups;
     std::vector<int32_t> kv_group_tasks;
     std::vector<WorkItem> fwd_items;
@@ -53,7 +60,7 @@ struct Schedule {
     int64_t partial_rows = 0;
     size_t bwd_workspace_bytes = 0;
     // byte offsets inside the backward workspace
-    size_t ws_dq_acc_off = 0, ws_delta_off = 0;
+    size_t ws_dq_acc_off = 0, ws_lse2_off = 0, ws_delta_off = 0;
 };
 
 // Validates the placement and fills `s`.  Pure host code, no CUDA.

@@ -61,7 +61,7 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
         if (len == 0) continue;
         Task t{};
         t.q_off = cu[i]; t.q_len = len; t.kv_off = cu[i]; t.kv_len = len;
-        t.partial_slot = -1; t.merge_group = -1; t.kv_group = -1; t.q_group = -1;
+        t.partial_slot = -1; t.q_slot = 0; t.kv_group = -1; t.q_group = -1;
         s->tasks.push_back(t);
         q_ranges.push_back({cu[i], len});
         kv_ranges.push_back({cu[i], len});
@@ -91,7 +91,7 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
         q_ranges.push_back({d.q_off, d.q_len});
         Task t{};
         t.q_off = d.q_off; t.q_len = d.q_len; t.kv_off = d.kv_off; t.kv_len = d.kv_len;
-        t.kv_group = -1; t.q_group = -1;
+        t.kv_group = -1; t.q_group = -1; t.q_slot = 0;
         auto mk = std::make_pair((int64_t)d.q_off, (int64_t)d.q_len);
         auto it = merge_index.find(mk);
         if (it == merge_index.end()) {
@@ -101,7 +101,6 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
         } else if (merge_seq[it->second] != d.seq_id) {
             return ZL_ERR_INVALID_ARG;
         }
-        t.merge_group = it->second;
         // slot padded to whole query tiles so a full-tile store of a ragged last tile can
         // never reach another task's slot
         const int32_t padded = (int32_t)align_up((size_t)d.q_len, kTileQ);
@@ -134,8 +133,14 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
             Task& t = s->tasks[ti];
             auto qk = std::make_pair((int64_t)t.q_off, (int64_t)t.q_len);
             auto qi = qg.find(qk);
-            if (qi == qg.end()) qi = qg.emplace(qk, (int32_t)qg.size()).first;
+            if (qi == qg.end()) {
+                qi = qg.emplace(qk, (int32_t)s->q_groups.size()).first;
+                const int32_t pad = (int32_t)align_up((size_t)t.q_len, kTileQ);
+                s->q_groups.push_back({t.q_off, t.q_len, (int32_t)s->q_pad_total, pad});
+                s->q_pad_total += pad;
+            }
             t.q_group = qi->second;
+            t.q_slot = s->q_groups[qi->second].slot;
             if (t.kv_len == 0) continue;
             auto kk = std::make_pair((int64_t)t.kv_off, (int64_t)t.kv_len);
             auto ki = kg.find(kk);
@@ -183,10 +188,14 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
         return std::tie(a.unit, a.head, a.row0) < std::tie(b.unit, b.head, b.row0);
     });
 
-    // backward workspace: fp32 dQ accumulator [total_q, H, d], then D [H, total_q]
+    // backward workspace over the padded query slots: fp32 dQ accumulator [q_pad, H, d], then
+    // LSE * log2(e) and D = rowsum(dO o O), both [H, q_pad]
+    if (s->q_pad_total > INT32_MAX) return ZL_ERR_INVALID_ARG;
+    const size_t vec_bytes = align_up((size_t)s->q_pad_total * n_heads * sizeof(float), 256);
     s->ws_dq_acc_off = 0;
-    s->ws_delta_off = align_up((size_t)total_q * n_heads * head_dim * sizeof(float), 256);
-    s->bwd_workspace_bytes = s->ws_delta_off + align_up((size_t)total_q * n_heads * sizeof(float), 256);
+    s->ws_lse2_off = align_up((size_t)s->q_pad_total * n_heads * head_dim * sizeof(float), 256);
+    s->ws_delta_off = s->ws_lse2_off + vec_bytes;
+    s->bwd_workspace_bytes = s->ws_delta_off + vec_bytes;
     return ZL_OK;
 }
 
