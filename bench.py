@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the coalesced attention engine on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--config 4] [--impl reference]
+
+A *step* is one pass of the whole hot path over one rank-local placement: the forward
+launch over whole sequences and shard tasks, the LSE merge, and the backward (preprocess,
+main, dQ conversion).  The task handle is built once per placement and reused, as a
+training loop reuses it for every layer.  Prints ONE JSON line (rank 0).
+
+  value     counted TFLOP/s of forward + backward (4*Lq*Lkv*d*H forward, 2.5x that
+            backward), inputs resident in HBM, device-timed with CUDA events
+  e2e       the same metric with pinned HOST buffers: every step copies Q, K, V, dO to the
+            device and O, LSE, dQ, dK, dV back, inside the timed region
+  roofline  the backward main kernel (dominant) against the measured dense bf16 peak
+  cpu_baseline  the fp64 CPU oracle timed on this machine's host cores on a bounded sample
+
+With N > 1 (torchrun) every rank runs its own rank-local placement of the same shape
+(weak scaling, no data-path collective); value is the sum over ranks divided by the
+slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "coalesced attention TFLOP/s fwd and fwd+bwd; % of B200 dense BF16 peak"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.path = tempfile.mktemp(prefix="zl_clocks_", suffix=".csv")
+        self.proc = None
+        try:
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=self.fh, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, mx, pw = [], [], []
+        reasons = set()
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [x.strip() for x in line.split(",")]
+                    if len(parts) < 8:
+                        continue
+                    try:
+                        sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+                    except ValueError:
+                        continue
+                    for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                        "sw_power_cap"), parts[4:8]):
+                        if v.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            # samples under load: upper half of the power readings
+            thr = statistics.median(pw) if pw else 0
+            under = [s for s, p in zip(sm, pw) if p >= thr] or sm
+            out.update(sm_mhz=statistics.median(under), sm_max_mhz=max(mx), samples=len(sm),
+                       power_w_max=max(pw) if pw else None)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# --------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------
+class Workload:
+    """Device tensors + task handle of one placement."""
+
+    def __init__(self, p, device, seed_shift=0):
+        import torch
+        import paper_2608_01150_b200 as Z
+        import zl_workloads as W
+        self.Z, self.p, self.torch = Z, p, torch
+        H, d = p.n_heads, p.head_dim
+        mk = lambda rows, s: W.device_normal_bf16((rows, H, d), p.seed * 100 + s + seed_shift, device)
+        self.Q, self.K, self.V, self.dO = mk(p.total_q, 0), mk(p.total_kv, 1), mk(p.total_kv, 2), mk(p.total_q, 3)
+        t0 = time.perf_counter()
+        self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, H, d)
+        self.build_ms = (time.perf_counter() - t0) * 1e3
+        info = self.h.info
+        self.O = torch.empty_like(self.Q)
+        self.LSE = torch.empty(H, p.total_q, dtype=torch.float32, device=device)
+        pr = max(1, int(info.partial_rows))
+        self.OP = torch.empty(pr, H, d, dtype=torch.float32, device=device)
+        self.LP = torch.empty(H, pr, dtype=torch.float32, device=device)
+        self.dQ, self.dK, self.dV = torch.empty_like(self.Q), torch.empty_like(self.K), torch.empty_like(self.V)
+        self.ws = torch.empty(max(256, int(info.bwd_workspace_bytes)), dtype=torch.uint8, device=device)
+        self.merge_bytes = (sum(s[1] for s in p.shards) * H * (d * 4 + 4)
+                            + sum(g[1] for g in {(s[0], s[1]) for s in p.shards}) * H * (d * 2 + 4))
+
+    def fwd(self):
+        Z, p = self.Z, self.p
+        Z.coalesced_attn_fwd(self.h, self.Q, self.K, self.V, p.scale, self.O, self.LSE, self.OP, self.LP)
+        Z.lse_merge(self.h, self.OP, self.LP, self.O, self.LSE)
+
+    def bwd(self):
+        self.Z.coalesced_attn_bwd(self.h, self.Q, self.K, self.V, self.O, self.LSE, self.dO, self.p.scale,
+                                  self.dQ, self.dK, self.dV, self.ws)
+
+    def step(self):
+        self.fwd()
+        self.bwd()
+
+    def time_region(self, fn, n, dist=None):
+        """Device time (ms) of n calls of fn, bracketed by barrier + synchronize; max over ranks."""
+        torch = self.torch
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], dtype=torch.float64, device=self.Q.device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dist.barrier()
+            ms = float(t.item())
+        return ms
+
+    def make_host_buffers(self):
+        torch = self.torch
+        pin = lambda t: torch.empty(t.shape, dtype=t.dtype, device="cpu", pin_memory=True).copy_(t)
+        self.hQ, self.hK, self.hV, self.hdO = pin(self.Q), pin(self.K), pin(self.V), pin(self.dO)
+        self.hO, self.hLSE = pin(self.O), pin(self.LSE)
+        self.hdQ, self.hdK, self.hdV = pin(self.dQ), pin(self.dK), pin(self.dV)
+        nb = lambda *ts: sum(t.numel() * t.element_size() for t in ts)
+        self.h2d_bytes = nb(self.hQ, self.hK, self.hV, self.hdO)
+        self.d2h_bytes = nb(self.hO, self.hLSE, self.hdQ, self.hdK, self.hdV)
+
+    def e2e_step(self):
+        for dst, src in ((self.Q, self.hQ), (self.K, self.hK), (self.V, self.hV), (self.dO, self.hdO)):
+            dst.copy_(src, non_blocking=True)
+        self.step()
+        for dst, src in ((self.hO, self.O), (self.hLSE, self.LSE), (self.hdQ, self.dQ), (self.hdK, self.dK),
+                         (self.hdV, self.dV)):
+            dst.copy_(src, non_blocking=True)
+
+
+def cpu_baseline(p, target_s=12.0):
+    """Times the fp64 CPU oracle (as it stands) on a bounded sample of the placement:
+    forward + backward of whole sequences / sampled query rows of the first heads."""
+    import numpy as np
+    import zl_workloads as W
+    from oracle import attention as A
+    cores = A.num_threads()
+    d = p.head_dim
+    rng = np.random.RandomState(0)
+    # sample problem: the first whole sequence of the placement (or 1024 rows of the first
+    # shard's query chunk against its full key set), head by head until the time target.
+    probs = A.logical_problems(p)
+    pr = probs[0]
+    n_q = min(pr["q_len"], 1560)
+    n_kv = sum(r[1] for r in pr["kv_ranges"])
+    flops_per_head = 3.5 * 4.0 * n_q * n_kv * d
+    t0 = time.perf_counter()
+    heads = 0
+    while True:
+        q = rng.standard_normal((n_q, d)); k = rng.standard_normal((n_kv, d))
+        v = rng.standard_normal((n_kv, d)); do = rng.standard_normal((n_q, d))
+        A.attn_bwd(q, k, v, do, p.scale)      # runs the oracle forward, then its backward
+        heads += 1
+        el = time.perf_counter() - t0
+        if el >= target_s or heads >= 4096:
+            break
+    return {"value": flops_per_head * heads / el / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+            "sample": f"{heads} head-problems of {n_q} query x {n_kv} key rows, d={d}, fwd+bwd in fp64 "
+                      f"({el:.1f} s), same FLOP convention",
+            "seconds": el}
+
+
+def run_ours(args):
+    import torch
+    import zl_workloads as W
+    import paper_2608_01150_b200 as Z
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    peaks, peak_kind = load_peaks()
+
+    p = W.config(args.config)
+    wl = Workload(p, device, seed_shift=rank * 7)
+    K, Wm = args.steps, max(3, args.warmup)
+    for _ in range(Wm):
+        wl.step()
+    torch.cuda.synchronize()
+    code, where = wl.h.last_device_status()
+    if code != 0:
+        raise RuntimeError(f"device status {code} at {where}")
+
+    uuid = str(torch.cuda.get_device_properties(device).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    launches0 = Z.launch_count()
+    ms_total = wl.time_region(wl.step, K, dist)
+    launches = Z.launch_count() - launches0
+    ms_fwd = wl.time_region(wl.fwd, K, dist)
+    clocks = sampler.stop()
+    ms_step = ms_total / K
+    flops = p.fwd_flops() + p.bwd_flops()
+    value = world * flops / (ms_step * 1e-3) / 1e12
+
+    # per-kernel device time (separate pass with event brackets around every launch)
+    wl.h.set_kernel_timing(True)
+    for _ in range(K):
+        wl.step()
+    kt = wl.h.get_kernel_timing()
+    wl.h.set_kernel_timing(False)
+    tot = sum(v[0] for v in kt.values()) or 1.0
+    kernels = {k: {"launches": v[1], "avg_ms": (v[0] / v[1] if v[1] else None), "share": v[0] / tot}
+               for k, v in kt.items()}
+    bm = kernels["bwd_main"]["avg_ms"]
+    peak_t = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    achieved = p.bwd_flops() / (bm * 1e-3) / 1e12 if bm else None
+    roofline = {"kernel": "zl_bwd_main_kernel", "bound": "tensor", "achieved": achieved, "peak": peak_t,
+                "unit": "TFLOP/s", "frac": (achieved / peak_t if achieved else None),
+                "peak_kind": f"{peak_kind} sustained bf16 (kernel timed inside a long step)",
+                "frac_of_burst": (achieved / float(peaks.get("bf16_tflops", 1590.0)) if achieved else None),
+                "traffic": None}
+    fm = kernels["fwd"]["avg_ms"]
+    fwd_kernel_tflops = p.fwd_flops() / (fm * 1e-3) / 1e12 if fm else None
+    mm = kernels["merge"]["avg_ms"]
+    merge_gbs = wl.merge_bytes / (mm * 1e-3) / 1e9 if mm else None
+
+    # end to end with host buffers
+    wl.make_host_buffers()
+    for _ in range(2):
+        wl.e2e_step()
+    ms_e2e = wl.time_region(wl.e2e_step, K, dist) / K
+    e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+           "h2d_bytes_per_step": wl.h2d_bytes, "d2h_bytes_per_step": wl.d2h_bytes}
+    code, where = wl.h.last_device_status()
+    if code != 0:
+        raise RuntimeError(f"device status {code} at {where}")
+
+    result = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": p.name, "n_heads": p.n_heads, "head_dim": p.head_dim, "total_q": p.total_q,
+                   "total_kv": p.total_kv, "tasks": int(wl.h.info.n_tasks),
+                   "step": "fwd launch + lse merge + bwd (pre, main, post)",
+                   "l2": "inputs larger than L2 (K+V alone exceed 126 MB); no flush",
+                   "parallelism": f"{world} independent rank-local placements"},
+        "fwd_tflops": world * p.fwd_flops() / (ms_fwd / K * 1e-3) / 1e12,
+        "fwd_ms": ms_fwd / K,
+        "frac_of_peak": {"burst_1645.7": value / world / float(peaks.get("bf16_tflops", 1590.0)),
+                         "sustained": value / world / peak_t, "datasheet_2250": value / world / 2250.0},
+        "build_tasks_ms": wl.build_ms,
+        "gpu_launches": int(launches),
+        "e2e": e2e, "roofline": roofline, "kernels": kernels,
+        "fwd_kernel_tflops": fwd_kernel_tflops, "merge_gbs": merge_gbs,
+        "merge_frac_of_hbm": (merge_gbs / float(peaks.get("hbm_gbs", 6650.0)) if merge_gbs else None),
+        "clocks": clocks,
+    }
+
+    if world == 1 and args.extra_configs:
+        extra = {}
+        del wl
+        torch.cuda.empty_cache()
+        for ci in [int(x) for x in args.extra_configs.split(",") if x]:
+            try:
+                pe = W.config(ci)
+                we = Workload(pe, device)
+                n = 3 if ci == 5 else 5
+                for _ in range(3):
+                    we.step()
+                tf = we.time_region(we.fwd, n) / n
+                tb = we.time_region(we.bwd, n) / n
+                extra[pe.name] = {"fwd_ms": tf, "bwd_ms": tb, "fwd_tflops": pe.fwd_flops() / tf / 1e9,
+                                  "bwd_tflops": pe.bwd_flops() / tb / 1e9,
+                                  "fwd_bwd_tflops": (pe.fwd_flops() + pe.bwd_flops()) / (tf + tb) / 1e9}
+                code, where = we.h.last_device_status()
+                if code != 0:
+                    extra[pe.name]["device_status"] = [code, where]
+                del we
+                torch.cuda.empty_cache()
+            except Exception as e:  # noqa: BLE001
+                extra[f"cfg{ci}"] = {"error": repr(e)}
+        result["per_config"] = extra
+
+    if world == 1 and rank == 0 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(p)
+    if rank == 0:
+        print(json.dumps(result), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------
+# reference arm: the fp64 CPU oracle on host cores
+# --------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import zl_workloads as W
+    p = W.config(args.config)
+    K, Wm = args.steps, max(1, min(args.warmup, 2))
+    per_step = max(1.0, min(8.0, 120.0 / (K + Wm)))
+    for _ in range(Wm):
+        cpu_baseline(p, target_s=per_step)
+    vals, secs, last = [], 0.0, None
+    for _ in range(K):
+        last = cpu_baseline(p, target_s=per_step)
+        vals.append(last["value"]); secs += last["seconds"]
+    v = sum(vals) / len(vals)
+    out = {"impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s",
+           "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": Wm,
+           "ms_per_step": secs / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "f64", "data": "synthetic",
+           "config": {"workload": p.name, "n_heads": p.n_heads, "head_dim": p.head_dim,
+                      "note": "each step is a bounded sample of the workload run by the fp64 CPU oracle"},
+           "cpu_baseline": {"value": v, "unit": "TFLOP/s", "kind": "oracle", "cores": last["cores"],
+                            "sample": last["sample"]},
+           "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4, help="named configuration 1..5 (default: Wan-14B-shaped rank)")
+    ap.add_argument("--extra-configs", default="2,3,5", help="also time these configurations (N=1 only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        port = 29500 + (os.getpid() % 2000)
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -163,6 +163,18 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* tasks, const void* q, const void
  * (kernel id * 1000 + site).  Resets the word to ZL_OK. */
 zl_status zl_last_device_status(const zl_tasks* tasks, int32_t* code, int32_t* where);
 
+/* Optional per-kernel device timing, for measurement only (no paper counterpart).  While
+ * enabled, every launch made through this handle is bracketed by CUDA events on the launch
+ * stream (at most 1024 launches per kernel between two reads; further ones are not timed).
+ * zl_get_kernel_timing synchronises the device, returns the summed elapsed milliseconds
+ * and the number of timed launches per kernel id, and clears the counters. */
+typedef enum {
+    ZL_K_FWD = 0, ZL_K_MERGE = 1, ZL_K_BWD_PRE = 2, ZL_K_BWD_MAIN = 3, ZL_K_BWD_POST = 4, ZL_K_COUNT = 5
+} zl_kernel_id;
+zl_status zl_set_kernel_timing(zl_tasks* tasks, int32_t enable);
+zl_status zl_get_kernel_timing(zl_tasks* tasks, float* total_ms /* [ZL_K_COUNT] */,
+                               int32_t* launches /* [ZL_K_COUNT] */);
+
 const char* zl_status_str(zl_status s);
 
 /* Number of this library's kernel launches enqueued since load (all handles). */

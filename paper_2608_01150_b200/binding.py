@@ -18,6 +18,9 @@ STATUS_NAMES = {0: "ZL_OK", 1: "ZL_ERR_INVALID_ARG", 2: "ZL_ERR_OVERLAP", 3: "ZL
                 4: "ZL_ERR_WORKSPACE", 5: "ZL_ERR_CUDA", 6: "ZL_ERR_TIMEOUT"}
 
 
+KERNEL_NAMES = ("fwd", "merge", "bwd_pre", "bwd_main", "bwd_post")
+
+
 class ZlError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
@@ -68,6 +71,10 @@ def _load():
                                           ctypes.c_size_t, vp]
     lib.zl_last_device_status.restype = ctypes.c_int
     lib.zl_last_device_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.zl_set_kernel_timing.restype = ctypes.c_int
+    lib.zl_set_kernel_timing.argtypes = [vp, i32]
+    lib.zl_get_kernel_timing.restype = ctypes.c_int
+    lib.zl_get_kernel_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.zl_status_str.restype = ctypes.c_char_p
     lib.zl_status_str.argtypes = [ctypes.c_int]
     lib.zl_launch_count.restype = ctypes.c_int64
@@ -142,6 +149,16 @@ class TaskHandle:
         c, w = ctypes.c_int32(), ctypes.c_int32()
         _check(_lib.zl_last_device_status(self._ptr, ctypes.byref(c), ctypes.byref(w)), "zl_last_device_status")
         return c.value, w.value
+
+    def set_kernel_timing(self, enable: bool):
+        _check(_lib.zl_set_kernel_timing(self._ptr, 1 if enable else 0), "zl_set_kernel_timing")
+
+    def get_kernel_timing(self):
+        """{kernel name: (total ms, launches)} since the last read; synchronises the device."""
+        ms = (ctypes.c_float * len(KERNEL_NAMES))()
+        n = (ctypes.c_int32 * len(KERNEL_NAMES))()
+        _check(_lib.zl_get_kernel_timing(self._ptr, ms, n), "zl_get_kernel_timing")
+        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(KERNEL_NAMES)}
 
     def close(self):
         if self._ptr:

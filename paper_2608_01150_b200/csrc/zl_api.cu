@@ -26,6 +26,10 @@ struct zl_tasks {
     KvGroup* d_kv_groups = nullptr;
     int32_t* d_kv_group_tasks = nullptr;
     int32_t* d_status = nullptr;
+    // optional per-kernel event timing (measurement only)
+    mutable bool timing = false;
+    mutable std::vector<cudaEvent_t> ev_start[ZL_K_COUNT], ev_stop[ZL_K_COUNT];
+    mutable int ev_used[ZL_K_COUNT] = {0, 0, 0, 0, 0};
 };
 
 namespace {
@@ -64,6 +68,30 @@ bool make_tmap(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int 
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
+
+constexpr int kMaxTimedLaunches = 1024;
+
+// Brackets one kernel launch with events when timing is enabled on the handle.
+struct LaunchTimer {
+    const zl_tasks* t;
+    int id;
+    cudaStream_t cs;
+    cudaEvent_t stop = nullptr;
+    LaunchTimer(const zl_tasks* t_, int id_, cudaStream_t cs_) : t(t_), id(id_), cs(cs_) {
+        if (!t->timing || t->ev_used[id] >= kMaxTimedLaunches) return;
+        const int i = t->ev_used[id];
+        if ((int)t->ev_start[id].size() <= i) {
+            cudaEvent_t a, b;
+            if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+            t->ev_start[id].push_back(a);
+            t->ev_stop[id].push_back(b);
+        }
+        cudaEventRecord(t->ev_start[id][i], cs);
+        stop = t->ev_stop[id][i];
+        t->ev_used[id] = i + 1;
+    }
+    ~LaunchTimer() { if (stop) cudaEventRecord(stop, cs); }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -211,6 +239,10 @@ zl_status zl_tasks_get_bwd_items(const zl_tasks* t, int32_t* items, int32_t capa
 
 void zl_free_tasks(zl_tasks* t) {
     if (!t) return;
+    for (int k = 0; k < ZL_K_COUNT; ++k) {
+        for (cudaEvent_t e : t->ev_start[k]) cudaEventDestroy(e);
+        for (cudaEvent_t e : t->ev_stop[k]) cudaEventDestroy(e);
+    }
     if (t->d_tables) cudaFree(t->d_tables);
     delete t;
 }
@@ -247,8 +279,11 @@ zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k,
     p.lse_partial = lse_partial;
     p.status = t->d_status;
     const int grid = std::min<int>(t->n_sms, p.n_items);
-    if (launch_fwd(s.head_dim, tq, tk, tv, p, grid, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-        return ZL_ERR_CUDA;
+    {
+        LaunchTimer lt(t, ZL_K_FWD, static_cast<cudaStream_t>(stream));
+        if (launch_fwd(s.head_dim, tq, tk, tv, p, grid, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return ZL_ERR_CUDA;
+    }
     g_launches.fetch_add(1);
     return ZL_OK;
 }
@@ -273,7 +308,11 @@ zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* l
     p.lse_partial = lse_partial;
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
-    if (launch_merge(s.head_dim, p, t->n_sms, static_cast<cudaStream_t>(stream)) != cudaSuccess) return ZL_ERR_CUDA;
+    {
+        LaunchTimer lt(t, ZL_K_MERGE, static_cast<cudaStream_t>(stream));
+        if (launch_merge(s.head_dim, p, t->n_sms, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return ZL_ERR_CUDA;
+    }
     g_launches.fetch_add(1);
     return ZL_OK;
 }
@@ -327,15 +366,45 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
 
     if (cudaMemsetAsync(p.dq_acc, 0, (size_t)s.q_pad_total * s.n_heads * s.head_dim * sizeof(float), cs) != cudaSuccess)
         return ZL_ERR_CUDA;
-    if (launch_bwd_pre(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+    {
+        LaunchTimer lt(t, ZL_K_BWD_PRE, cs);
+        if (launch_bwd_pre(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+    }
     g_launches.fetch_add(1);
     if (p.n_items > 0) {
         const int grid = std::min<int>(t->n_sms, p.n_items);
+        LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
         if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
         g_launches.fetch_add(1);
     }
-    if (launch_bwd_post(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+    {
+        LaunchTimer lt(t, ZL_K_BWD_POST, cs);
+        if (launch_bwd_post(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+    }
     g_launches.fetch_add(1);
+    return ZL_OK;
+}
+
+zl_status zl_set_kernel_timing(zl_tasks* t, int32_t enable) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    t->timing = enable != 0;
+    return ZL_OK;
+}
+
+zl_status zl_get_kernel_timing(zl_tasks* t, float* total_ms, int32_t* launches) {
+    if (!t || !total_ms || !launches) return ZL_ERR_INVALID_ARG;
+    for (int k = 0; k < ZL_K_COUNT; ++k) { total_ms[k] = 0.f; launches[k] = 0; }
+    if (t->device < 0) return ZL_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) return ZL_ERR_CUDA;
+    for (int k = 0; k < ZL_K_COUNT; ++k) {
+        for (int i = 0; i < t->ev_used[k]; ++i) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, t->ev_start[k][i], t->ev_stop[k][i]) != cudaSuccess) return ZL_ERR_CUDA;
+            total_ms[k] += ms;
+        }
+        launches[k] = t->ev_used[k];
+        t->ev_used[k] = 0;
+    }
     return ZL_OK;
 }
 
