@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -92,6 +93,20 @@ struct LaunchTimer {
     }
     ~LaunchTimer() { if (stop) cudaEventRecord(stop, cs); }
 };
+
+// Tensor map over the fp32 dQ accumulator [rows, H, d]: box = 32 columns x 1 head x 128 rows.
+bool make_tmap_f32_acc(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)(rows > 0 ? rows : 1)};
+    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 4, (cuuint64_t)head_dim * 4 * n_heads};
+    cuuint32_t box[3] = {32, 1, 128};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -332,14 +347,15 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     if (workspace_bytes < s.bwd_workspace_bytes) return ZL_ERR_WORKSPACE;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
-    CUtensorMap tq, tk, tv, tdo;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    CUtensorMap tq, tk, tv, tdo, tdq;
+    if (!make_tmap_f32_acc(&tdq, ws + s.ws_dq_acc_off, s.q_pad_total, s.n_heads, s.head_dim)) return ZL_ERR_CUDA;
     if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ) ||
         !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
         !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
         !make_tmap(&tdo, d_o, s.total_q, s.n_heads, s.head_dim, kTileQ))
         return ZL_ERR_CUDA;
 
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
     BwdParams p{};
     p.tasks = t->d_tasks;
     p.items = t->d_bwd_items;
@@ -353,6 +369,10 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     p.q_pad_total = (int32_t)s.q_pad_total;
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
+    {
+        const char* e = getenv("ZL_DQ_MODE");
+        p.dq_mode = e ? atoi(e) : 1;
+    }
     p.o = static_cast<const __nv_bfloat16*>(o);
     p.d_o = static_cast<const __nv_bfloat16*>(d_o);
     p.lse = lse;
@@ -374,7 +394,7 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     if (p.n_items > 0) {
         const int grid = std::min<int>(t->n_sms, p.n_items);
         LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
-        if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
+        if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, tdq, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
         g_launches.fetch_add(1);
     }
     {

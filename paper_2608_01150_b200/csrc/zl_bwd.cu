@@ -106,24 +106,28 @@ __global__ void __launch_bounds__(kPreThreads) zl_bwd_post_kernel(const BwdParam
 }
 
 // ======================================================================= main
-constexpr int kBwdThreads = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 P/dS, warps 6-9 dQ
+// Warp roles (16 warps): warp 0 TMA producer, warp 1 MMA issuer, warps 2-3 idle,
+// warps 4-7 and 8-11 two P/dS warpgroups (query columns 0-63 and 64-127 of every tile, one key
+// row per thread), warps 12-15 dQ warpgroup (one query row per thread).
+constexpr int kBwdThreads = 512;
 
 template <int D>
 struct BwdSmem {
-    static constexpr int kStages = (D == 128) ? 1 : 2;
     static constexpr int kTileBytes = 128 * D * 2;
     static constexpr int kBoxBytes = 128 * 128;
     static constexpr int kBoxes = D / 64;
+    static constexpr int kDqChunkBytes = 128 * 32 * 4;  // 128 query rows x 32 fp32 columns
     alignas(1024) uint8_t k[kTileBytes];
     alignas(1024) uint8_t v[kTileBytes];
-    alignas(1024) uint8_t q[kStages][kTileBytes];
-    alignas(1024) uint8_t d_o[kStages][kTileBytes];
-    alignas(1024) uint8_t ds[2 * kBoxBytes];  // dS^T tile: 128 key rows x 128 query columns, bf16
-    alignas(16) float lse2[kStages][128];
-    alignas(16) float delta[kStages][128];
+    alignas(1024) uint8_t q[2][kTileBytes];
+    alignas(1024) uint8_t d_o[kTileBytes];
+    alignas(1024) uint8_t ds[2 * kBoxBytes];            // dS^T tile: 128 key rows x 128 query columns, bf16
+    alignas(1024) uint8_t dq_stage[2][kDqChunkBytes];   // fp32 dQ chunks staged for the TMA reduce
+    alignas(16) float lse2[2][128];
+    alignas(16) float delta[2][128];
     alignas(8) uint64_t kv_full, kv_empty;
-    uint64_t qdo_full[kStages], qdo_empty[kStages];
-    uint64_t s_full, p_full, ds_full, dq_full, dq_empty, acc_full;
+    uint64_t q_full[2], q_empty[2], do_full, do_empty;
+    uint64_t s_full, dp_full, p_full, ds_full, dq_full, dq_empty, acc_full;
     uint32_t tmem_base;
     volatile int32_t abort_flag;
 };
@@ -149,16 +153,23 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
         }                                                                            \
     } while (0)
 
+// Number of 128-row query tiles a kv group's CTA iterates over.
+__device__ __forceinline__ int count_q_tiles(const BwdParams& p, const KvGroup& g) {
+    int n = 0;
+    for (int ti = 0; ti < g.n_tasks; ++ti)
+        n += (p.tasks[p.kv_group_tasks[g.task_begin + ti]].q_len + kTileQ - 1) / kTileQ;
+    return n;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                   const BwdParams p) {
+                   const __grid_constant__ CUtensorMap tm_dq, const BwdParams p) {
     using Smem = BwdSmem<D>;
-    constexpr int kStages = Smem::kStages;
     constexpr int kBoxes = Smem::kBoxes;
-    extern __shared__ uint8_t smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -166,16 +177,23 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // TMEM columns: S^T / P^T [0,128), dP^T / dQ [128,256), dV [256,256+D), dK [384,384+D)
     constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384, kTmemCols = 512;
 
+    if ((smem_u32(smem_raw) & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
+        if (threadIdx.x == 0 && atomicCAS(p.status, 0, (int)ZL_ERR_CUDA) == 0) p.status[1] = 2999;
+        return;
+    }
     if (threadIdx.x == 0) {
         mbar_init(&sm.kv_full, 1);
         mbar_init(&sm.kv_empty, 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.qdo_full[s], 1);
-            mbar_init(&sm.qdo_empty[s], 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&sm.q_full[s], 1);
+            mbar_init(&sm.q_empty[s], 1);
         }
+        mbar_init(&sm.do_full, 1);
+        mbar_init(&sm.do_empty, 1);
         mbar_init(&sm.s_full, 1);
-        mbar_init(&sm.p_full, 128);
-        mbar_init(&sm.ds_full, 128);
+        mbar_init(&sm.dp_full, 1);
+        mbar_init(&sm.p_full, 256);
+        mbar_init(&sm.ds_full, 256);
         mbar_init(&sm.dq_full, 1);
         mbar_init(&sm.dq_empty, 128);
         mbar_init(&sm.acc_full, 1);
@@ -185,6 +203,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
         prefetch_tmap(&tm_do);
+        prefetch_tmap(&tm_dq);
     }
     if (warp == 1) {
         tmem_alloc(&sm.tmem_base, kTmemCols);
@@ -195,9 +214,10 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+    if (warp < 4) {
+        reg_dec<72>();
+        if (warp == 0 && lane == 0) {
+            // -------------------------------------------------------------- TMA producer
             uint32_t item_cnt = 0, it_cnt = 0;
             for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
                 const WorkItem wi = p.items[it];
@@ -212,90 +232,110 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                     const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
                     for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
-                        const int s = it_cnt % kStages;
-                        ZL_WAIT(&sm.qdo_empty[s], ((it_cnt / kStages) & 1) ^ 1, 2);
-                        mbar_arrive_expect_tx(&sm.qdo_full[s], 2 * Smem::kTileBytes + 1024);
-                        for (int b = 0; b < kBoxes; ++b) {
-                            tma_load_3d(sm.q[s] + b * Smem::kBoxBytes, &tm_q, &sm.qdo_full[s], b * 64, wi.head,
+                        const int s = it_cnt & 1;
+                        ZL_WAIT(&sm.q_empty[s], ((it_cnt >> 1) & 1) ^ 1, 2);
+                        mbar_arrive_expect_tx(&sm.q_full[s], Smem::kTileBytes + 1024);
+                        for (int b = 0; b < kBoxes; ++b)
+                            tma_load_3d(sm.q[s] + b * Smem::kBoxBytes, &tm_q, &sm.q_full[s], b * 64, wi.head,
                                         t.q_off + qt * kTileQ);
-                            tma_load_3d(sm.d_o[s] + b * Smem::kBoxBytes, &tm_do, &sm.qdo_full[s], b * 64, wi.head,
-                                        t.q_off + qt * kTileQ);
-                        }
                         const int64_t vec = (int64_t)wi.head * p.q_pad_total + t.q_slot + qt * kTileQ;
-                        bulk_load_1d(sm.lse2[s], p.lse2 + vec, 512, &sm.qdo_full[s]);
-                        bulk_load_1d(sm.delta[s], p.delta + vec, 512, &sm.qdo_full[s]);
+                        bulk_load_1d(sm.lse2[s], p.lse2 + vec, 512, &sm.q_full[s]);
+                        bulk_load_1d(sm.delta[s], p.delta + vec, 512, &sm.q_full[s]);
+                        ZL_WAIT(&sm.do_empty, (it_cnt & 1) ^ 1, 3);
+                        mbar_arrive_expect_tx(&sm.do_full, Smem::kTileBytes);
+                        for (int b = 0; b < kBoxes; ++b)
+                            tma_load_3d(sm.d_o + b * Smem::kBoxBytes, &tm_do, &sm.do_full, b * 64, wi.head,
+                                        t.q_off + qt * kTileQ);
                     }
                 }
             }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        } else if (warp == 1 && lane == 0) {
+            // -------------------------------------------------------------- MMA issuer
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: K-major x K-major
             constexpr uint32_t idesc_dv = make_idesc_bf16(128, D, 0, 1);    // A in TMEM / K-major smem, B MN-major
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 1, 1);    // A MN-major smem, B MN-major
             const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v), ds_addr = smem_u32(sm.ds);
+            const uint32_t do_addr = smem_u32(sm.d_o);
+            auto issue_s = [&](uint32_t q_addr) {
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
+                    mma_ss(tmem + kColS, make_desc_sw128(k_addr + off, 16, 1024),
+                           make_desc_sw128(q_addr + off, 16, 1024), idesc_s, ks > 0);
+                }
+                mma_commit(&sm.s_full);
+            };
+            auto issue_dp = [&]() {
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
+                    mma_ss(tmem + kColDP, make_desc_sw128(v_addr + off, 16, 1024),
+                           make_desc_sw128(do_addr + off, 16, 1024), idesc_s, ks > 0);
+                }
+                mma_commit(&sm.dp_full);
+            };
             uint32_t item_cnt = 0, it_cnt = 0;
             for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
+                const int n_it = count_q_tiles(p, g);
                 ZL_WAIT(&sm.kv_full, item_cnt & 1, 11);
-                bool first = true;
-                for (int ti = 0; ti < g.n_tasks; ++ti) {
-                    const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
-                    const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
-                    for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
-                        const int s = it_cnt % kStages;
-                        const uint32_t q_addr = smem_u32(sm.q[s]), do_addr = smem_u32(sm.d_o[s]);
-                        ZL_WAIT(&sm.qdo_full[s], (it_cnt / kStages) & 1, 12);
-                        ZL_WAIT(&sm.dq_empty, (it_cnt & 1) ^ 1, 13);  // previous dQ tile drained
+                // prologue: S and dP of the item's first query tile
+                ZL_WAIT(&sm.q_full[it_cnt & 1], (it_cnt >> 1) & 1, 12);
+                tc_fence_after();
+                issue_s(smem_u32(sm.q[it_cnt & 1]));
+                ZL_WAIT(&sm.do_full, it_cnt & 1, 13);
+                ZL_WAIT(&sm.dq_empty, (it_cnt & 1) ^ 1, 14);  // previous dQ tile drained from the dP columns
+                tc_fence_after();
+                issue_dp();
+                for (int i = 0; i < n_it; ++i, ++it_cnt) {
+                    const uint32_t q_addr = smem_u32(sm.q[it_cnt & 1]);
+                    const bool has_next = i + 1 < n_it;
+                    const uint32_t nxt = it_cnt + 1;
+                    ZL_WAIT(&sm.p_full, it_cnt & 1, 15);
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
+                        mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8,
+                               make_desc_sw128(do_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, i > 0 || ks > 0);
+                    mma_commit(&sm.do_empty);
+                    if (has_next) {
+                        ZL_WAIT(&sm.q_full[nxt & 1], (nxt >> 1) & 1, 16);
                         tc_fence_after();
+                        issue_s(smem_u32(sm.q[nxt & 1]));  // overwrites P^T(i): ordered after dV(i) on the tensor pipe
+                    }
+                    ZL_WAIT(&sm.ds_full, it_cnt & 1, 17);
+                    tc_fence_after();
 #pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks) {
-                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                            mma_ss(tmem + kColS, make_desc_sw128(k_addr + off, 16, 1024),
-                                   make_desc_sw128(q_addr + off, 16, 1024), idesc_s, ks > 0);
-                        }
+                    for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
+                        const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
+                        mma_ss(tmem + kColDK, make_desc_sw128(ds_addr + off, 16, 1024),
+                               make_desc_sw128(q_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, i > 0 || ks > 0);
+                    }
 #pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks) {
-                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                            mma_ss(tmem + kColDP, make_desc_sw128(v_addr + off, 16, 1024),
-                                   make_desc_sw128(do_addr + off, 16, 1024), idesc_s, ks > 0);
-                        }
-                        mma_commit(&sm.s_full);
-                        ZL_WAIT(&sm.p_full, it_cnt & 1, 14);
+                    for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
+                        mma_ss(tmem + kColDP, make_desc_sw128(ds_addr + ks * 2048, Smem::kBoxBytes, 1024),
+                               make_desc_sw128(k_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dq, ks > 0);
+                    mma_commit(&sm.dq_full);
+                    mma_commit(&sm.q_empty[it_cnt & 1]);
+                    if (has_next) {
+                        ZL_WAIT(&sm.do_full, nxt & 1, 18);
+                        ZL_WAIT(&sm.dq_empty, it_cnt & 1, 19);
                         tc_fence_after();
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
-                            mma_ts(tmem + kColDV, tmem + kColS + ks * 8,
-                                   make_desc_sw128(do_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv,
-                                   !first || ks > 0);
-                        ZL_WAIT(&sm.ds_full, it_cnt & 1, 15);
-                        tc_fence_after();
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
-                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                            mma_ss(tmem + kColDK, make_desc_sw128(ds_addr + off, 16, 1024),
-                                   make_desc_sw128(q_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv,
-                                   !first || ks > 0);
-                        }
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows
-                            mma_ss(tmem + kColDP, make_desc_sw128(ds_addr + ks * 2048, Smem::kBoxBytes, 1024),
-                                   make_desc_sw128(k_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dq, ks > 0);
-                        mma_commit(&sm.dq_full);
-                        mma_commit(&sm.qdo_empty[s]);
-                        first = false;
+                        issue_dp();
                     }
                 }
                 mma_commit(&sm.acc_full);
                 mma_commit(&sm.kv_empty);
             }
         }
-    } else if (warp < 6) {
-        // ------------------------------------------------------------------ P / dS warps (one key row per thread)
+    } else if (warp < 12) {
+        // ------------------------------------------------------------------ P / dS warpgroups
+        reg_inc<168>();
+        const int wg = (warp - 4) >> 2;            // 0: query columns 0-63, 1: columns 64-127
         const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;
+        const int row = quarter * 32 + lane;       // key row within the tile
+        const int col0 = wg * 64;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const uint32_t ds_row_addr = smem_u32(sm.ds) + row * 128;
         const float sl2 = p.scale_log2;
@@ -308,78 +348,85 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                 const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
-                    const int s = it_cnt % kStages;
+                    const int s = it_cnt & 1;
                     const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
-                    ZL_WAIT_WARP(&sm.qdo_full[s], (it_cnt / kStages) & 1, 21);  // lse2 / delta vectors
-                    ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 22);
-                    if (it_cnt > 0) ZL_WAIT_WARP(&sm.dq_full, (it_cnt - 1) & 1, 23);  // dS buffer consumed
-                    tc_fence_after();
                     const bool full = row_ok && q_valid == kTileQ;
+                    ZL_WAIT_WARP(&sm.q_full[s], (it_cnt >> 1) & 1, 21);  // lse2 / delta vectors
+                    ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 22);
+                    tc_fence_after();
+                    float pv[64];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t sr[32], dr[32];
-                        tmem_ld_x32(lane_addr + kColS + c * 32, sr);
-                        tmem_ld_x32(lane_addr + kColDP + c * 32, dr);
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t sr[32];
+                        tmem_ld_x32(lane_addr + kColS + col0 + c * 32, sr);
                         tmem_wait_ld();
-                        uint32_t pp[16], dd[16];
+                        uint32_t pp[16];
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            const int col = c * 32 + i;
+                            const int col = col0 + c * 32 + i;
                             const float2 l2 = *reinterpret_cast<const float2*>(&sm.lse2[s][col]);
-                            const float2 dl = *reinterpret_cast<const float2*>(&sm.delta[s][col]);
                             float p0 = ex2(fmaf(__uint_as_float(sr[i]), sl2, -l2.x));
                             float p1 = ex2(fmaf(__uint_as_float(sr[i + 1]), sl2, -l2.y));
-                            float d0 = p0 * (__uint_as_float(dr[i]) - dl.x);
-                            float d1 = p1 * (__uint_as_float(dr[i + 1]) - dl.y);
                             if (!full) {
-                                const bool ok0 = row_ok && col < q_valid, ok1 = row_ok && col + 1 < q_valid;
-                                p0 = ok0 ? p0 : 0.f; d0 = ok0 ? d0 : 0.f;
-                                p1 = ok1 ? p1 : 0.f; d1 = ok1 ? d1 : 0.f;
+                                p0 = (row_ok && col < q_valid) ? p0 : 0.f;
+                                p1 = (row_ok && col + 1 < q_valid) ? p1 : 0.f;
                             }
+                            pv[c * 32 + i] = p0;
+                            pv[c * 32 + i + 1] = p1;
                             pp[i / 2] = pack_bf16(p0, p1);
-                            dd[i / 2] = pack_bf16(d0, d1);
                         }
-                        tmem_st_x16(lane_addr + kColS + c * 16, pp);
-#pragma unroll
-                        for (int k4 = 0; k4 < 4; ++k4) {
-                            const int c16 = c * 4 + k4;  // 16-byte chunk index along the query axis
-                            const uint32_t addr = ds_row_addr + (c16 >> 3) * Smem::kBoxBytes + (((c16 & 7) ^ (row & 7)) << 4);
-                            st_shared_v4(addr, dd[k4 * 4], dd[k4 * 4 + 1], dd[k4 * 4 + 2], dd[k4 * 4 + 3]);
-                        }
+                        tmem_st_x16(lane_addr + kColS + col0 + c * 16, pp);
                     }
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(&sm.p_full);
+
+                    ZL_WAIT_WARP(&sm.dp_full, it_cnt & 1, 23);
+                    if (it_cnt > 0) ZL_WAIT_WARP(&sm.dq_full, (it_cnt - 1) & 1, 24);  // dS buffer consumed
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t dr[32];
+                        tmem_ld_x32(lane_addr + kColDP + col0 + c * 32, dr);
+                        tmem_wait_ld();
+                        uint32_t dd[16];
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            const int col = col0 + c * 32 + i;
+                            const float2 dl = *reinterpret_cast<const float2*>(&sm.delta[s][col]);
+                            float d0 = pv[c * 32 + i] * (__uint_as_float(dr[i]) - dl.x);
+                            float d1 = pv[c * 32 + i + 1] * (__uint_as_float(dr[i + 1]) - dl.y);
+                            if (!full) {
+                                d0 = (row_ok && col < q_valid) ? d0 : 0.f;
+                                d1 = (row_ok && col + 1 < q_valid) ? d1 : 0.f;
+                            }
+                            dd[i / 2] = pack_bf16(d0, d1);
+                        }
+#pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            const int c16 = (col0 >> 3) + c * 4 + k4;  // 16-byte chunk index along the query axis
+                            const uint32_t addr = ds_row_addr + (c16 >> 3) * Smem::kBoxBytes + (((c16 & 7) ^ (row & 7)) << 4);
+                            st_shared_v4(addr, dd[k4 * 4], dd[k4 * 4 + 1], dd[k4 * 4 + 2], dd[k4 * 4 + 3]);
+                        }
+                    }
+                    tc_fence_before();
                     fence_proxy_async_smem();
                     mbar_arrive(&sm.ds_full);
                 }
             }
-            // ---- epilogue: dV and dK of this key tile
-            ZL_WAIT_WARP(&sm.acc_full, item_cnt & 1, 24);
+            // ---- epilogue: warpgroup 0 stores dV, warpgroup 1 stores dK (scaled)
+            ZL_WAIT_WARP(&sm.acc_full, item_cnt & 1, 25);
             tc_fence_after();
             const int64_t grow = (int64_t)g.kv_off + wi.row0 + row;
-            __nv_bfloat16* dv_dst = p.dv + (grow * p.n_heads + wi.head) * D;
-            __nv_bfloat16* dk_dst = p.dk + (grow * p.n_heads + wi.head) * D;
+            __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + (grow * p.n_heads + wi.head) * D;
+            const float sc = (wg == 0) ? 1.f : p.scale;
+            const uint32_t col_acc = (wg == 0) ? kColDV : kColDK;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld_x32(lane_addr + kColDV + c * 32, r);
+                tmem_ld_x32(lane_addr + col_acc + c * 32, r);
                 tmem_wait_ld();
                 if (row_ok) {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 o4;
-                        o4.x = pack_bf16(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                        o4.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                        o4.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-                        o4.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-                        *reinterpret_cast<uint4*>(dv_dst + c * 32 + i) = o4;
-                    }
-                }
-                tmem_ld_x32(lane_addr + kColDK + c * 32, r);
-                tmem_wait_ld();
-                if (row_ok) {
-                    const float sc = p.scale;
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         uint4 o4;
@@ -387,18 +434,20 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         o4.y = pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc);
                         o4.z = pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc);
                         o4.w = pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc);
-                        *reinterpret_cast<uint4*>(dk_dst + c * 32 + i) = o4;
+                        *reinterpret_cast<uint4*>(dst + c * 32 + i) = o4;
                     }
                 }
             }
             tc_fence_before();
         }
     } else {
-        // ------------------------------------------------------------------ dQ warps (one query row per thread)
+        // ------------------------------------------------------------------ dQ warpgroup (one query row per thread)
+        reg_dec<104>();
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-        uint32_t it_cnt = 0;
+        const bool leader = (warp == 12 && lane == 0);
+        uint32_t it_cnt = 0, chunk_cnt = 0;
         for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
             const WorkItem wi = p.items[it];
             const KvGroup g = p.kv_groups[wi.unit];
@@ -406,30 +455,61 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                 const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
-                    const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
                     ZL_WAIT_WARP(&sm.dq_full, it_cnt & 1, 31);
                     tc_fence_after();
-                    float* dst = p.dq_acc + (((int64_t)t.q_slot + qt * kTileQ + row) * p.n_heads + wi.head) * D;
-                    uint32_t r[D];
+                    if (p.dq_mode == 0) {
+                        // vector reductions straight from registers
+                        const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
+                        float* dst = p.dq_acc + (((int64_t)t.q_slot + qt * kTileQ + row) * p.n_heads + wi.head) * D;
 #pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t tmp[32];
-                        tmem_ld_x32(lane_addr + kColDP + c * 32, tmp);
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t r[32];
+                            tmem_ld_x32(lane_addr + kColDP + c * 32, r);
+                            tmem_wait_ld();
+                            if (c == D / 32 - 1) {
+                                tc_fence_before();
+                                mbar_arrive(&sm.dq_empty);
+                            }
+                            if (row < q_valid) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[c * 32 + i] = tmp[i];
-                    }
-                    tmem_wait_ld();
-                    tc_fence_before();
-                    mbar_arrive(&sm.dq_empty);
-                    if (row < q_valid) {
+                                for (int i = 0; i < 32; i += 4)
+                                    red_add_v4(dst + c * 32 + i, __uint_as_float(r[i]), __uint_as_float(r[i + 1]),
+                                               __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                            }
+                        }
+                    } else {
+                        // stage 32-column chunks in swizzled shared memory, add them with the TMA
+#pragma unroll 1
+                        for (int c = 0; c < D / 32; ++c, ++chunk_cnt) {
+                            uint8_t* buf = sm.dq_stage[chunk_cnt & 1];
+                            if (chunk_cnt >= 2) {
+                                if (leader) bulk_wait_group_read<1>();  // the reduce that last read this buffer is done
+                                named_bar_sync(1, 128);
+                            }
+                            uint32_t r[32];
+                            tmem_ld_x32(lane_addr + kColDP + c * 32, r);
+                            tmem_wait_ld();
+                            if (c == D / 32 - 1) {
+                                tc_fence_before();
+                                mbar_arrive(&sm.dq_empty);
+                            }
+                            const uint32_t row_addr = smem_u32(buf) + row * 128;
 #pragma unroll
-                        for (int i = 0; i < D; i += 4)
-                            red_add_v4(dst + i, __uint_as_float(r[i]), __uint_as_float(r[i + 1]),
-                                       __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                            for (int k4 = 0; k4 < 8; ++k4)
+                                st_shared_v4(row_addr + ((k4 ^ (row & 7)) << 4), r[k4 * 4], r[k4 * 4 + 1], r[k4 * 4 + 2],
+                                             r[k4 * 4 + 3]);
+                            fence_proxy_async_smem();
+                            named_bar_sync(1, 128);
+                            if (leader) {
+                                tma_reduce_add_3d(&tm_dq, buf, c * 32, wi.head, t.q_slot + qt * kTileQ);
+                                bulk_commit_group();
+                            }
+                        }
                     }
                 }
             }
         }
+        if (leader) bulk_wait_group<0>();
     }
 
 teardown:
@@ -444,15 +524,16 @@ teardown:
 
 template <int D>
 cudaError_t launch_main_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                          const CUtensorMap& tdo, const BwdParams& p, int grid, cudaStream_t stream) {
-    constexpr int smem = sizeof(BwdSmem<D>) + 1024;
+                          const CUtensorMap& tdo, const CUtensorMap& tdq, const BwdParams& p, int grid,
+                          cudaStream_t stream) {
+    constexpr int smem = sizeof(BwdSmem<D>);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(zl_bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    zl_bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, p);
+    zl_bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, tdq, p);
     return cudaGetLastError();
 }
 
@@ -467,10 +548,11 @@ cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStre
 }
 
 cudaError_t launch_bwd_main(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                            const CUtensorMap& tdo, const BwdParams& p, int grid, cudaStream_t stream) {
+                            const CUtensorMap& tdo, const CUtensorMap& tdq, const BwdParams& p, int grid,
+                            cudaStream_t stream) {
     if (p.n_items == 0) return cudaSuccess;
-    return head_dim == 128 ? launch_main_t<128>(tq, tk, tv, tdo, p, grid, stream)
-                           : launch_main_t<64>(tq, tk, tv, tdo, p, grid, stream);
+    return head_dim == 128 ? launch_main_t<128>(tq, tk, tv, tdo, tdq, p, grid, stream)
+                           : launch_main_t<64>(tq, tk, tv, tdo, tdq, p, grid, stream);
 }
 
 cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream) {

@@ -51,6 +51,7 @@ struct BwdParams {
     int32_t q_pad_total;
     float scale;
     float scale_log2;
+    int32_t dq_mode;  // 0: vector reductions from registers, 1: TMA reduce-add from shared memory
     const __nv_bfloat16* o;
     const __nv_bfloat16* d_o;
     const float* lse;
@@ -65,7 +66,8 @@ struct BwdParams {
 
 cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
 cudaError_t launch_bwd_main(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                            const CUtensorMap& tdo, const BwdParams& p, int grid, cudaStream_t stream);
+                            const CUtensorMap& tdo, const CUtensorMap& tdq, const BwdParams& p, int grid,
+                            cudaStream_t stream);
 cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
 
 cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
