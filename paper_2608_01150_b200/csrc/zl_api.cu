@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -384,6 +385,14 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     p.delta = reinterpret_cast<float*>(ws + s.ws_delta_off);
     p.status = t->d_status;
 
+#ifdef ZL_PROFILE
+    static long long* d_prof = nullptr;
+    if (getenv("ZL_PROF")) {
+        if (!d_prof) cudaMalloc(&d_prof, 4 * 64 * sizeof(long long));
+        cudaMemsetAsync(d_prof, 0, 4 * 64 * sizeof(long long), cs);
+        p.prof = d_prof;
+    }
+#endif
     if (cudaMemsetAsync(p.dq_acc, 0, (size_t)s.q_pad_total * s.n_heads * s.head_dim * sizeof(float), cs) != cudaSuccess)
         return ZL_ERR_CUDA;
     {
@@ -402,6 +411,18 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
         if (launch_bwd_post(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
     }
     g_launches.fetch_add(1);
+#ifdef ZL_PROFILE
+    if (p.prof) {
+        long long hprof[4 * 64];
+        cudaStreamSynchronize(cs);
+        cudaMemcpy(hprof, p.prof, sizeof(hprof), cudaMemcpyDeviceToHost);
+        for (int b = 0; b < 2; ++b) {
+            fprintf(stderr, "[zl prof] cta %d total %lld :", b, hprof[b * 64]);
+            for (int i = 1; i < 64; ++i) if (hprof[b * 64 + i]) fprintf(stderr, " s%d=%lld", i, hprof[b * 64 + i]);
+            fprintf(stderr, "\n");
+        }
+    }
+#endif
     return ZL_OK;
 }
 

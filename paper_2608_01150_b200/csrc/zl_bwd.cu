@@ -127,7 +127,7 @@ struct BwdSmem {
     alignas(16) float delta[2][128];
     alignas(8) uint64_t kv_full, kv_empty;
     uint64_t q_full[2], q_empty[2], do_full, do_empty;
-    uint64_t s_full, dp_full, p_full, ds_full, dq_full, dq_empty, acc_full;
+    uint64_t s_full, dp_full, p_full, ds_full, ds_free, dq_full, dq_empty, acc_full;
     uint32_t tmem_base;
     volatile int32_t abort_flag;
 };
@@ -137,20 +137,40 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
     if (atomicCAS(status, 0, (int)ZL_ERR_TIMEOUT) == 0) status[1] = where;
 }
 
+#ifdef ZL_PROFILE
+// Development aid (profile builds only): cycles spent waiting at each site and in each MMA
+// issue segment, for the first CTAs.
+#define ZL_PROF_T0 const long long prof_t0_ = clock64();
+#define ZL_PROF_ADD(site) \
+    if (p.prof && blockIdx.x < 4 && lane == 0) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_t0_));
+#define ZL_PROF_SEG_BEGIN const long long prof_seg_ = clock64();
+#define ZL_PROF_SEG_END(site) \
+    if (p.prof && blockIdx.x < 4) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_seg_));
+#else
+#define ZL_PROF_T0
+#define ZL_PROF_ADD(site)
+#define ZL_PROF_SEG_BEGIN
+#define ZL_PROF_SEG_END(site)
+#endif
+
 #define ZL_WAIT(bar, parity, site)                                        \
     do {                                                                  \
+        ZL_PROF_T0                                                        \
         if (!mbar_wait((bar), (parity), kWaitLimitNs) || sm.abort_flag) { \
             report(p.status, &sm.abort_flag, 2000 + (site));              \
             goto teardown;                                                \
         }                                                                 \
+        ZL_PROF_ADD(site)                                                 \
     } while (0)
 #define ZL_WAIT_WARP(bar, parity, site)                                              \
     do {                                                                             \
+        ZL_PROF_T0                                                                   \
         const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs) && !sm.abort_flag; \
         if (!__all_sync(0xffffffffu, ok_)) {                                         \
             report(p.status, &sm.abort_flag, 2000 + (site));                         \
             goto teardown;                                                           \
         }                                                                            \
+        if (warp == 4 || warp == 12) { ZL_PROF_ADD(site) }                           \
     } while (0)
 
 // Number of 128-row query tiles a kv group's CTA iterates over.
@@ -194,6 +214,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mbar_init(&sm.dp_full, 1);
         mbar_init(&sm.p_full, 256);
         mbar_init(&sm.ds_full, 256);
+        mbar_init(&sm.ds_free, 1);
         mbar_init(&sm.dq_full, 1);
         mbar_init(&sm.dq_empty, 128);
         mbar_init(&sm.acc_full, 1);
@@ -213,9 +234,12 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
+#ifdef ZL_PROFILE
+    const long long prof_start = clock64();
+#endif
 
     if (warp < 4) {
-        reg_dec<72>();
+        reg_dec<80>();
         if (warp == 0 && lane == 0) {
             // -------------------------------------------------------------- TMA producer
             uint32_t item_cnt = 0, it_cnt = 0;
@@ -257,6 +281,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v), ds_addr = smem_u32(sm.ds);
             const uint32_t do_addr = smem_u32(sm.d_o);
             auto issue_s = [&](uint32_t q_addr) {
+                ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
@@ -264,8 +289,10 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                            make_desc_sw128(q_addr + off, 16, 1024), idesc_s, ks > 0);
                 }
                 mma_commit(&sm.s_full);
+                ZL_PROF_SEG_END(40)
             };
             auto issue_dp = [&]() {
+                ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
@@ -273,6 +300,16 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                            make_desc_sw128(do_addr + off, 16, 1024), idesc_s, ks > 0);
                 }
                 mma_commit(&sm.dp_full);
+                ZL_PROF_SEG_END(41)
+            };
+            auto issue_dv = [&](bool acc) {
+                ZL_PROF_SEG_BEGIN
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
+                    mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8,
+                           make_desc_sw128(do_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, acc || ks > 0);
+                mma_commit(&sm.do_empty);
+                ZL_PROF_SEG_END(42)
             };
             uint32_t item_cnt = 0, it_cnt = 0;
             for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
@@ -280,7 +317,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const KvGroup g = p.kv_groups[wi.unit];
                 const int n_it = count_q_tiles(p, g);
                 ZL_WAIT(&sm.kv_full, item_cnt & 1, 11);
-                // prologue: S and dP of the item's first query tile
+                // prologue: S, dP, dV of the item's first query tile and S of the second.
+                // Steady-state order on the tensor pipe: dQ(i) dK(i) dP(i+1) dV(i+1) S(i+2).
                 ZL_WAIT(&sm.q_full[it_cnt & 1], (it_cnt >> 1) & 1, 12);
                 tc_fence_after();
                 issue_s(smem_u32(sm.q[it_cnt & 1]));
@@ -288,41 +326,50 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ZL_WAIT(&sm.dq_empty, (it_cnt & 1) ^ 1, 14);  // previous dQ tile drained from the dP columns
                 tc_fence_after();
                 issue_dp();
+                ZL_WAIT(&sm.p_full, it_cnt & 1, 15);
+                tc_fence_after();
+                issue_dv(false);
+                if (n_it > 1) {
+                    const uint32_t n1 = it_cnt + 1;
+                    ZL_WAIT(&sm.q_full[n1 & 1], (n1 >> 1) & 1, 16);
+                    tc_fence_after();
+                    issue_s(smem_u32(sm.q[n1 & 1]));  // overwrites P^T: ordered after dV on the tensor pipe
+                }
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     const uint32_t q_addr = smem_u32(sm.q[it_cnt & 1]);
-                    const bool has_next = i + 1 < n_it;
-                    const uint32_t nxt = it_cnt + 1;
-                    ZL_WAIT(&sm.p_full, it_cnt & 1, 15);
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
-                        mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8,
-                               make_desc_sw128(do_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, i > 0 || ks > 0);
-                    mma_commit(&sm.do_empty);
-                    if (has_next) {
-                        ZL_WAIT(&sm.q_full[nxt & 1], (nxt >> 1) & 1, 16);
-                        tc_fence_after();
-                        issue_s(smem_u32(sm.q[nxt & 1]));  // overwrites P^T(i): ordered after dV(i) on the tensor pipe
-                    }
                     ZL_WAIT(&sm.ds_full, it_cnt & 1, 17);
                     tc_fence_after();
+                    {
+                        ZL_PROF_SEG_BEGIN
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
-                        const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                        mma_ss(tmem + kColDK, make_desc_sw128(ds_addr + off, 16, 1024),
-                               make_desc_sw128(q_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, i > 0 || ks > 0);
+                        for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
+                            mma_ss(tmem + kColDP, make_desc_sw128(ds_addr + ks * 2048, Smem::kBoxBytes, 1024),
+                                   make_desc_sw128(k_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dq, ks > 0);
+                        mma_commit(&sm.dq_full);
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
+                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
+                            mma_ss(tmem + kColDK, make_desc_sw128(ds_addr + off, 16, 1024),
+                                   make_desc_sw128(q_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, i > 0 || ks > 0);
+                        }
+                        mma_commit(&sm.q_empty[it_cnt & 1]);
+                        mma_commit(&sm.ds_free);
+                        ZL_PROF_SEG_END(43)
                     }
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
-                        mma_ss(tmem + kColDP, make_desc_sw128(ds_addr + ks * 2048, Smem::kBoxBytes, 1024),
-                               make_desc_sw128(k_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dq, ks > 0);
-                    mma_commit(&sm.dq_full);
-                    mma_commit(&sm.q_empty[it_cnt & 1]);
-                    if (has_next) {
-                        ZL_WAIT(&sm.do_full, nxt & 1, 18);
+                    if (i + 1 < n_it) {
+                        const uint32_t n1 = it_cnt + 1, n2 = it_cnt + 2;
+                        ZL_WAIT(&sm.do_full, n1 & 1, 18);
                         ZL_WAIT(&sm.dq_empty, it_cnt & 1, 19);
                         tc_fence_after();
                         issue_dp();
+                        ZL_WAIT(&sm.p_full, n1 & 1, 20);
+                        tc_fence_after();
+                        issue_dv(true);
+                        if (i + 2 < n_it) {
+                            ZL_WAIT(&sm.q_full[n2 & 1], (n2 >> 1) & 1, 16);
+                            tc_fence_after();
+                            issue_s(smem_u32(sm.q[n2 & 1]));
+                        }
                     }
                 }
                 mma_commit(&sm.acc_full);
@@ -331,7 +378,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
     } else if (warp < 12) {
         // ------------------------------------------------------------------ P / dS warpgroups
-        reg_inc<168>();
+        reg_inc<128>();
         const int wg = (warp - 4) >> 2;            // 0: query columns 0-63, 1: columns 64-127
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;       // key row within the tile
@@ -354,7 +401,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ZL_WAIT_WARP(&sm.q_full[s], (it_cnt >> 1) & 1, 21);  // lse2 / delta vectors
                     ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 22);
                     tc_fence_after();
-                    float pv[64];
+                    uint32_t pk[32];  // P^T of this thread's row, bf16 pairs
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
                         uint32_t sr[32];
@@ -371,9 +418,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                 p0 = (row_ok && col < q_valid) ? p0 : 0.f;
                                 p1 = (row_ok && col + 1 < q_valid) ? p1 : 0.f;
                             }
-                            pv[c * 32 + i] = p0;
-                            pv[c * 32 + i + 1] = p1;
                             pp[i / 2] = pack_bf16(p0, p1);
+                            pk[c * 16 + i / 2] = pp[i / 2];
                         }
                         tmem_st_x16(lane_addr + kColS + col0 + c * 16, pp);
                     }
@@ -382,7 +428,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     mbar_arrive(&sm.p_full);
 
                     ZL_WAIT_WARP(&sm.dp_full, it_cnt & 1, 23);
-                    if (it_cnt > 0) ZL_WAIT_WARP(&sm.dq_full, (it_cnt - 1) & 1, 24);  // dS buffer consumed
+                    if (it_cnt > 0) ZL_WAIT_WARP(&sm.ds_free, (it_cnt - 1) & 1, 24);  // dS buffer consumed by dK/dQ
                     tc_fence_after();
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
@@ -394,8 +440,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         for (int i = 0; i < 32; i += 2) {
                             const int col = col0 + c * 32 + i;
                             const float2 dl = *reinterpret_cast<const float2*>(&sm.delta[s][col]);
-                            float d0 = pv[c * 32 + i] * (__uint_as_float(dr[i]) - dl.x);
-                            float d1 = pv[c * 32 + i + 1] * (__uint_as_float(dr[i + 1]) - dl.y);
+                            const uint32_t pw = pk[c * 16 + i / 2];
+                            float d0 = __uint_as_float(pw << 16) * (__uint_as_float(dr[i]) - dl.x);
+                            float d1 = __uint_as_float(pw & 0xffff0000u) * (__uint_as_float(dr[i + 1]) - dl.y);
                             if (!full) {
                                 d0 = (row_ok && col < q_valid) ? d0 : 0.f;
                                 d1 = (row_ok && col + 1 < q_valid) ? d1 : 0.f;
@@ -442,7 +489,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
     } else {
         // ------------------------------------------------------------------ dQ warpgroup (one query row per thread)
-        reg_dec<104>();
+        reg_inc<176>();
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
@@ -478,26 +525,31 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             }
                         }
                     } else {
-                        // stage 32-column chunks in swizzled shared memory, add them with the TMA
-#pragma unroll 1
+                        // read the whole tile (frees the TMEM columns for the next dP^T), then stage
+                        // 32-column chunks in swizzled shared memory and add them with the TMA
+                        uint32_t r[D];
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t tmp[32];
+                            tmem_ld_x32(lane_addr + kColDP + c * 32, tmp);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) r[c * 32 + i] = tmp[i];
+                        }
+                        tmem_wait_ld();
+                        tc_fence_before();
+                        mbar_arrive(&sm.dq_empty);
+#pragma unroll
                         for (int c = 0; c < D / 32; ++c, ++chunk_cnt) {
                             uint8_t* buf = sm.dq_stage[chunk_cnt & 1];
                             if (chunk_cnt >= 2) {
                                 if (leader) bulk_wait_group_read<1>();  // the reduce that last read this buffer is done
                                 named_bar_sync(1, 128);
                             }
-                            uint32_t r[32];
-                            tmem_ld_x32(lane_addr + kColDP + c * 32, r);
-                            tmem_wait_ld();
-                            if (c == D / 32 - 1) {
-                                tc_fence_before();
-                                mbar_arrive(&sm.dq_empty);
-                            }
                             const uint32_t row_addr = smem_u32(buf) + row * 128;
 #pragma unroll
                             for (int k4 = 0; k4 < 8; ++k4)
-                                st_shared_v4(row_addr + ((k4 ^ (row & 7)) << 4), r[k4 * 4], r[k4 * 4 + 1], r[k4 * 4 + 2],
-                                             r[k4 * 4 + 3]);
+                                st_shared_v4(row_addr + ((k4 ^ (row & 7)) << 4), r[c * 32 + k4 * 4], r[c * 32 + k4 * 4 + 1],
+                                             r[c * 32 + k4 * 4 + 2], r[c * 32 + k4 * 4 + 3]);
                             fence_proxy_async_smem();
                             named_bar_sync(1, 128);
                             if (leader) {
@@ -513,6 +565,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
 
 teardown:
+#ifdef ZL_PROFILE
+    if (p.prof && blockIdx.x < 4 && threadIdx.x == 32) p.prof[blockIdx.x * 64 + 0] = clock64() - prof_start;
+#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {

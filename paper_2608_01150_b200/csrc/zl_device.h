@@ -62,6 +62,7 @@ struct BwdParams {
     float* lse2;    // [H, q_pad_total]: lse * log2(e), +inf on padding rows
     float* delta;   // [H, q_pad_total]: rowsum(dO o O), 0 on padding rows
     int32_t* status;
+    long long* prof;  // development aid (ZL_PROFILE builds), else null
 };
 
 cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
