@@ -381,8 +381,7 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     p.dk = static_cast<__nv_bfloat16*>(dk);
     p.dv = static_cast<__nv_bfloat16*>(dv);
     p.dq_acc = reinterpret_cast<float*>(ws + s.ws_dq_acc_off);
-    p.lse2 = reinterpret_cast<float*>(ws + s.ws_lse2_off);
-    p.delta = reinterpret_cast<float*>(ws + s.ws_delta_off);
+    p.aug = ws + s.ws_aug_off;
     p.status = t->d_status;
 
 #ifdef ZL_PROFILE

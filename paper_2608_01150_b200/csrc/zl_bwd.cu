@@ -7,8 +7,11 @@
 //     D_i = sum_c dO_ic O_ic.
 //
 // Three launches:
-//   pre   D and LSE*log2(e) into padded per-query-range scratch rows (the dQ accumulator is
-//         cleared by a memset node before it);
+//   pre   per 128-row query tile and head, a 4 KB "augmentation" tile holding -LSE/scale and
+//         -D, each split into three bf16 pieces (the dQ accumulator is cleared by a memset node
+//         before it).  The main kernel appends one extra K=16 MMA step to S^T and to dP^T whose
+//         A operand is a tile of ones, so the tensor core itself produces S^T - LSE/scale and
+//         dP^T - D: no per-column vector has to be broadcast from shared memory;
 //   main  persistent; a CTA owns one 128-row key tile of one kv group and one head, keeps
 //         K, V in shared memory and dK, dV in TMEM, and loops over every 128-row query tile
 //         of every task that shares the key range.  Per tile it issues five tcgen05 MMAs
@@ -40,18 +43,31 @@ __device__ __forceinline__ int find_q_group(const QGroup* g, int n, int slot_row
     return lo;
 }
 
+// Splits x into three bf16 pieces whose sum reproduces x to about 24 bits.
+__device__ __forceinline__ void split3(float x, __nv_bfloat16 (&h)[3]) {
+    h[0] = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(h[0]);
+    h[1] = __float2bfloat16_rn(r1);
+    h[2] = __float2bfloat16_rn(r1 - __bfloat162float(h[1]));
+}
+
+// Augmentation tile layout (4 KB per 128 query rows, K-major without swizzle): element e (0..15)
+// of row r lives at byte (e/8)*2048 + (r/8)*128 + (r%8)*16 + (e%8)*2.  Elements 0..2 hold the
+// pieces of -LSE/scale, elements 8..10 the pieces of -D, everything else is zero.  Rows past the
+// end of the query range get -1e30 and 0, which makes their P and dS vanish.
 template <int D>
 __global__ void __launch_bounds__(kPreThreads) zl_bwd_pre_kernel(const BwdParams p) {
     constexpr int V = D / 32;
     const int lane = threadIdx.x & 31;
     const int64_t n_units = (int64_t)p.q_pad_total * p.n_heads;
+    const float inv_scale = 1.f / p.scale;
     for (int64_t u = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); u < n_units;
          u += (int64_t)gridDim.x * (kPreThreads / 32)) {
         const int slot_row = (int)(u / p.n_heads);
         const int h = (int)(u - (int64_t)slot_row * p.n_heads);
         const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, slot_row)];
         const int r = slot_row - g.slot;
-        float delta = 0.f, l2 = INFINITY;
+        float xd = 0.f, xl = -1e30f;
         if (r < g.q_len) {
             const int64_t row = (int64_t)g.q_off + r;
             const __nv_bfloat16* po = p.o + (row * p.n_heads + h) * D + lane * V;
@@ -66,13 +82,21 @@ __global__ void __launch_bounds__(kPreThreads) zl_bwd_pre_kernel(const BwdParams
             }
 #pragma unroll
             for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-            delta = acc;
+            xd = -acc;
             const float l = p.lse[(int64_t)h * p.total_q + row];
-            l2 = (l == -INFINITY) ? INFINITY : l * 1.4426950408889634f;
+            if (l > -INFINITY && l < INFINITY) xl = -l * inv_scale;
         }
-        if (lane == 0) {
-            p.delta[(int64_t)h * p.q_pad_total + slot_row] = delta;
-            p.lse2[(int64_t)h * p.q_pad_total + slot_row] = l2;
+        // lanes 0..15 write the 16 bf16 elements of this row (32 bytes in two 16-byte halves)
+        if (lane < 16) {
+            __nv_bfloat16 hl[3], hd[3];
+            split3(xl, hl);
+            split3(xd, hd);
+            __nv_bfloat16 val = __float2bfloat16_rn(0.f);
+            if (lane < 3) val = hl[lane];
+            else if (lane >= 8 && lane < 11) val = hd[lane - 8];
+            const int tile = slot_row / kTileQ, tr = slot_row % kTileQ;
+            uint8_t* base = p.aug + ((int64_t)h * (p.q_pad_total / kTileQ) + tile) * 4096;
+            *reinterpret_cast<__nv_bfloat16*>(base + (lane / 8) * 2048 + (tr / 8) * 128 + (tr % 8) * 16 + (lane % 8) * 2) = val;
         }
     }
 }
@@ -122,9 +146,9 @@ struct BwdSmem {
     alignas(1024) uint8_t q[2][kTileBytes];
     alignas(1024) uint8_t d_o[kTileBytes];
     alignas(1024) uint8_t ds[2 * kBoxBytes];            // dS^T tile: 128 key rows x 128 query columns, bf16
-    alignas(1024) uint8_t dq_stage[2][kDqChunkBytes];   // fp32 dQ chunks staged for the TMA reduce
-    alignas(16) float lse2[2][128];
-    alignas(16) float delta[2][128];
+    alignas(1024) uint8_t dq_stage[kDqChunkBytes];      // one fp32 dQ chunk staged for the TMA reduce
+    alignas(1024) uint8_t aug[2][4096];                 // per Q stage: bf16 pieces of -LSE/scale and -D
+    alignas(1024) uint8_t ones[3][2048];                // [zeros][ones in elements 0..2][zeros]
     alignas(8) uint64_t kv_full, kv_empty;
     uint64_t q_full[2], q_empty[2], do_full, do_empty;
     uint64_t s_full, dp_full, p_full, ds_full, ds_free, dq_full, dq_empty, acc_full;
@@ -226,6 +250,14 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         prefetch_tmap(&tm_do);
         prefetch_tmap(&tm_dq);
     }
+    // constant A operand of the augmentation steps: 128 rows x 8 bf16 per block
+    for (int i = threadIdx.x; i < 3 * 2048 / 4; i += kBwdThreads) {
+        const int blk = i / 512, w = i % 4;  // w: 32-bit word inside the row's 16 bytes
+        uint32_t val = 0;
+        if (blk == 1) val = (w == 0) ? 0x3F803F80u : (w == 1 ? 0x00003F80u : 0u);
+        reinterpret_cast<uint32_t*>(&sm.ones[0][0])[i] = val;
+    }
+    fence_proxy_async_smem();
     if (warp == 1) {
         tmem_alloc(&sm.tmem_base, kTmemCols);
         tmem_relinquish();
@@ -258,13 +290,12 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
                         const int s = it_cnt & 1;
                         ZL_WAIT(&sm.q_empty[s], ((it_cnt >> 1) & 1) ^ 1, 2);
-                        mbar_arrive_expect_tx(&sm.q_full[s], Smem::kTileBytes + 1024);
+                        mbar_arrive_expect_tx(&sm.q_full[s], Smem::kTileBytes + 4096);
                         for (int b = 0; b < kBoxes; ++b)
                             tma_load_3d(sm.q[s] + b * Smem::kBoxBytes, &tm_q, &sm.q_full[s], b * 64, wi.head,
                                         t.q_off + qt * kTileQ);
-                        const int64_t vec = (int64_t)wi.head * p.q_pad_total + t.q_slot + qt * kTileQ;
-                        bulk_load_1d(sm.lse2[s], p.lse2 + vec, 512, &sm.q_full[s]);
-                        bulk_load_1d(sm.delta[s], p.delta + vec, 512, &sm.q_full[s]);
+                        const int64_t tile = (int64_t)wi.head * (p.q_pad_total / kTileQ) + t.q_slot / kTileQ + qt;
+                        bulk_load_1d(sm.aug[s], p.aug + tile * 4096, 4096, &sm.q_full[s]);
                         ZL_WAIT(&sm.do_empty, (it_cnt & 1) ^ 1, 3);
                         mbar_arrive_expect_tx(&sm.do_full, Smem::kTileBytes);
                         for (int b = 0; b < kBoxes; ++b)
@@ -280,18 +311,24 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 1, 1);    // A MN-major smem, B MN-major
             const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v), ds_addr = smem_u32(sm.ds);
             const uint32_t do_addr = smem_u32(sm.d_o);
-            auto issue_s = [&](uint32_t q_addr) {
+            const uint32_t ones_addr = smem_u32(&sm.ones[0][0]);
+            // S^T = K Q^T - LSE/scale: the last step multiplies the ones block with the LSE pieces
+            auto issue_s = [&](uint32_t stage) {
                 ZL_PROF_SEG_BEGIN
+                const uint32_t q_addr = smem_u32(sm.q[stage]);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
                     mma_ss(tmem + kColS, make_desc_sw128(k_addr + off, 16, 1024),
                            make_desc_sw128(q_addr + off, 16, 1024), idesc_s, ks > 0);
                 }
+                mma_ss(tmem + kColS, make_desc_noswizzle(ones_addr + 2048, 2048, 128),
+                       make_desc_noswizzle(smem_u32(sm.aug[stage]), 2048, 128), idesc_s, true);
                 mma_commit(&sm.s_full);
                 ZL_PROF_SEG_END(40)
             };
-            auto issue_dp = [&]() {
+            // dP^T = V dO^T - D: the ones sit in the second K chunk, where the tile holds the D pieces
+            auto issue_dp = [&](uint32_t stage) {
                 ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
@@ -299,6 +336,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     mma_ss(tmem + kColDP, make_desc_sw128(v_addr + off, 16, 1024),
                            make_desc_sw128(do_addr + off, 16, 1024), idesc_s, ks > 0);
                 }
+                mma_ss(tmem + kColDP, make_desc_noswizzle(ones_addr, 2048, 128),
+                       make_desc_noswizzle(smem_u32(sm.aug[stage]), 2048, 128), idesc_s, true);
                 mma_commit(&sm.dp_full);
                 ZL_PROF_SEG_END(41)
             };
@@ -321,11 +360,11 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 // Steady-state order on the tensor pipe: dQ(i) dK(i) dP(i+1) dV(i+1) S(i+2).
                 ZL_WAIT(&sm.q_full[it_cnt & 1], (it_cnt >> 1) & 1, 12);
                 tc_fence_after();
-                issue_s(smem_u32(sm.q[it_cnt & 1]));
+                issue_s(it_cnt & 1);
                 ZL_WAIT(&sm.do_full, it_cnt & 1, 13);
                 ZL_WAIT(&sm.dq_empty, (it_cnt & 1) ^ 1, 14);  // previous dQ tile drained from the dP columns
                 tc_fence_after();
-                issue_dp();
+                issue_dp(it_cnt & 1);
                 ZL_WAIT(&sm.p_full, it_cnt & 1, 15);
                 tc_fence_after();
                 issue_dv(false);
@@ -333,7 +372,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const uint32_t n1 = it_cnt + 1;
                     ZL_WAIT(&sm.q_full[n1 & 1], (n1 >> 1) & 1, 16);
                     tc_fence_after();
-                    issue_s(smem_u32(sm.q[n1 & 1]));  // overwrites P^T: ordered after dV on the tensor pipe
+                    issue_s(n1 & 1);  // overwrites P^T: ordered after dV on the tensor pipe
                 }
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     const uint32_t q_addr = smem_u32(sm.q[it_cnt & 1]);
@@ -361,14 +400,14 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         ZL_WAIT(&sm.do_full, n1 & 1, 18);
                         ZL_WAIT(&sm.dq_empty, it_cnt & 1, 19);
                         tc_fence_after();
-                        issue_dp();
+                        issue_dp(n1 & 1);
                         ZL_WAIT(&sm.p_full, n1 & 1, 20);
                         tc_fence_after();
                         issue_dv(true);
                         if (i + 2 < n_it) {
                             ZL_WAIT(&sm.q_full[n2 & 1], (n2 >> 1) & 1, 16);
                             tc_fence_after();
-                            issue_s(smem_u32(sm.q[n2 & 1]));
+                            issue_s(n2 & 1);
                         }
                     }
                 }
@@ -395,10 +434,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                 const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
-                    const int s = it_cnt & 1;
                     const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
                     const bool full = row_ok && q_valid == kTileQ;
-                    ZL_WAIT_WARP(&sm.q_full[s], (it_cnt >> 1) & 1, 21);  // lse2 / delta vectors
                     ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 22);
                     tc_fence_after();
                     uint32_t pk[32];  // P^T of this thread's row, bf16 pairs
@@ -411,9 +448,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
                             const int col = col0 + c * 32 + i;
-                            const float2 l2 = *reinterpret_cast<const float2*>(&sm.lse2[s][col]);
-                            float p0 = ex2(fmaf(__uint_as_float(sr[i]), sl2, -l2.x));
-                            float p1 = ex2(fmaf(__uint_as_float(sr[i + 1]), sl2, -l2.y));
+                            float p0 = ex2(__uint_as_float(sr[i]) * sl2);      // S^T already has -LSE/scale folded in
+                            float p1 = ex2(__uint_as_float(sr[i + 1]) * sl2);
                             if (!full) {
                                 p0 = (row_ok && col < q_valid) ? p0 : 0.f;
                                 p1 = (row_ok && col + 1 < q_valid) ? p1 : 0.f;
@@ -439,10 +475,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
                             const int col = col0 + c * 32 + i;
-                            const float2 dl = *reinterpret_cast<const float2*>(&sm.delta[s][col]);
                             const uint32_t pw = pk[c * 16 + i / 2];
-                            float d0 = __uint_as_float(pw << 16) * (__uint_as_float(dr[i]) - dl.x);
-                            float d1 = __uint_as_float(pw & 0xffff0000u) * (__uint_as_float(dr[i + 1]) - dl.y);
+                            float d0 = __uint_as_float(pw << 16) * __uint_as_float(dr[i]);           // dP^T already has -D
+                            float d1 = __uint_as_float(pw & 0xffff0000u) * __uint_as_float(dr[i + 1]);
                             if (!full) {
                                 d0 = (row_ok && col < q_valid) ? d0 : 0.f;
                                 d1 = (row_ok && col + 1 < q_valid) ? d1 : 0.f;
@@ -540,9 +575,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         mbar_arrive(&sm.dq_empty);
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c, ++chunk_cnt) {
-                            uint8_t* buf = sm.dq_stage[chunk_cnt & 1];
-                            if (chunk_cnt >= 2) {
-                                if (leader) bulk_wait_group_read<1>();  // the reduce that last read this buffer is done
+                            uint8_t* buf = sm.dq_stage;
+                            if (chunk_cnt >= 1) {
+                                if (leader) bulk_wait_group_read<0>();  // the previous reduce has read the buffer
                                 named_bar_sync(1, 128);
                             }
                             const uint32_t row_addr = smem_u32(buf) + row * 128;

@@ -59,8 +59,7 @@ struct BwdParams {
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     float* dq_acc;  // [q_pad_total, H, d]
-    float* lse2;    // [H, q_pad_total]: lse * log2(e), +inf on padding rows
-    float* delta;   // [H, q_pad_total]: rowsum(dO o O), 0 on padding rows
+    uint8_t* aug;   // [H, q_pad_total / 128] tiles of 4 KB: bf16 splits of -lse/scale and -rowsum(dO o O)
     int32_t* status;
     long long* prof;  // development aid (ZL_PROFILE builds), else null
 };

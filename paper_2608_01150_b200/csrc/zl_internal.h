@@ -60,7 +60,7 @@ struct Schedule {
     int64_t partial_rows = 0;
     size_t bwd_workspace_bytes = 0;
     // byte offsets inside the backward workspace
-    size_t ws_dq_acc_off = 0, ws_lse2_off = 0, ws_delta_off = 0;
+    size_t ws_dq_acc_off = 0, ws_aug_off = 0;
 };
 
 // Validates the placement and fills `s`.  Pure host code, no CUDA.

@@ -164,6 +164,18 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t smem_addr, uint32_t
     return d;
 }
 
+// Same format without swizzle (layout type 0), K-major: a core matrix is 8 rows x 16 bytes stored
+// contiguously (128 B); SBO = byte distance between 8-row groups, LBO = byte distance between the
+// two 8-element K chunks of one K=16 step.
+__device__ __forceinline__ uint64_t make_desc_noswizzle(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+
 // Instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
 //   bits [4,6) D format = 1 (f32); [7,10) A format = 1 (bf16); [10,13) B format = 1 (bf16)
 //   bit 15 A major (0 = K, 1 = MN); bit 16 B major; bits [17,23) N >> 3; bits [24,29) M >> 4

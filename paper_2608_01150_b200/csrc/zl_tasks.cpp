@@ -188,14 +188,13 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
         return std::tie(a.unit, a.head, a.row0) < std::tie(b.unit, b.head, b.row0);
     });
 
-    // backward workspace over the padded query slots: fp32 dQ accumulator [q_pad, H, d], then
-    // LSE * log2(e) and D = rowsum(dO o O), both [H, q_pad]
+    // backward workspace over the padded query slots: fp32 dQ accumulator [q_pad, H, d], then one
+    // 4 KB "augmentation" tile per (head, 128-row query tile) holding -LSE/scale and -D split
+    // into bf16 pieces (see the backward preprocess kernel)
     if (s->q_pad_total > INT32_MAX) return ZL_ERR_INVALID_ARG;
-    const size_t vec_bytes = align_up((size_t)s->q_pad_total * n_heads * sizeof(float), 256);
     s->ws_dq_acc_off = 0;
-    s->ws_lse2_off = align_up((size_t)s->q_pad_total * n_heads * head_dim * sizeof(float), 256);
-    s->ws_delta_off = s->ws_lse2_off + vec_bytes;
-    s->bwd_workspace_bytes = s->ws_delta_off + vec_bytes;
+    s->ws_aug_off = align_up((size_t)s->q_pad_total * n_heads * head_dim * sizeof(float), 256);
+    s->bwd_workspace_bytes = s->ws_aug_off + align_up((size_t)(s->q_pad_total / kTileQ) * n_heads * 4096, 256);
     return ZL_OK;
 }
 
