@@ -387,8 +387,8 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
 #ifdef ZL_PROFILE
     static long long* d_prof = nullptr;
     if (getenv("ZL_PROF")) {
-        if (!d_prof) cudaMalloc(&d_prof, 4 * 64 * sizeof(long long));
-        cudaMemsetAsync(d_prof, 0, 4 * 64 * sizeof(long long), cs);
+        if (!d_prof) cudaMalloc(&d_prof, 1024 * sizeof(long long));
+        cudaMemsetAsync(d_prof, 0, 1024 * sizeof(long long), cs);
         p.prof = d_prof;
     }
 #endif
@@ -412,13 +412,25 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     g_launches.fetch_add(1);
 #ifdef ZL_PROFILE
     if (p.prof) {
-        long long hprof[4 * 64];
+        long long hprof[1024];
         cudaStreamSynchronize(cs);
         cudaMemcpy(hprof, p.prof, sizeof(hprof), cudaMemcpyDeviceToHost);
         for (int b = 0; b < 2; ++b) {
             fprintf(stderr, "[zl prof] cta %d total %lld :", b, hprof[b * 64]);
             for (int i = 1; i < 64; ++i) if (hprof[b * 64 + i]) fprintf(stderr, " s%d=%lld", i, hprof[b * 64 + i]);
             fprintf(stderr, "\n");
+        }
+        if (getenv("ZL_TRACE")) {
+            const long long t0 = hprof[256 + 0];
+            for (int role = 0; role < 3; ++role)
+                for (int itx = 0; itx < 8; ++itx) {
+                    fprintf(stderr, "[zl trace] role %d it %d:", role, 200 + itx);
+                    for (int ev = 0; ev < 11; ++ev) {
+                        const long long v = hprof[256 + role * 128 + itx * 16 + ev];
+                        if (v) fprintf(stderr, " e%d=%lld", ev, v - t0);
+                    }
+                    fprintf(stderr, "\n");
+                }
         }
     }
 #endif

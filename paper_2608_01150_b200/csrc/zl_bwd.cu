@@ -167,6 +167,12 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 #define ZL_PROF_T0 const long long prof_t0_ = clock64();
 #define ZL_PROF_ADD(site) \
     if (p.prof && blockIdx.x < 4 && lane == 0) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_t0_));
+#define ZL_PROF_MARK(site) \
+    if (p.prof && blockIdx.x < 4 && warp == 4 && lane == 0) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_seg_));
+// Event trace: timestamp of event `ev` (0..15) of role `role` (0 MMA, 1 P/dS warp 4, 2 dQ warp 12) for
+// global iterations 200..207 of CTA 0.
+#define ZL_TRACE(role, ev, itc) \
+    if (p.prof && blockIdx.x == 0 && (itc) >= 200u && (itc) < 208u) p.prof[256 + (role) * 128 + ((itc) - 200u) * 16 + (ev)] = clock64();
 #define ZL_PROF_SEG_BEGIN const long long prof_seg_ = clock64();
 #define ZL_PROF_SEG_END(site) \
     if (p.prof && blockIdx.x < 4) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_seg_));
@@ -175,6 +181,8 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 #define ZL_PROF_ADD(site)
 #define ZL_PROF_SEG_BEGIN
 #define ZL_PROF_SEG_END(site)
+#define ZL_PROF_MARK(site)
+#define ZL_TRACE(role, ev, itc)
 #endif
 
 #define ZL_WAIT(bar, parity, site)                                        \
@@ -271,7 +279,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #endif
 
     if (warp < 4) {
-        reg_dec<80>();
+        reg_dec<104>();
         if (warp == 0 && lane == 0) {
             // -------------------------------------------------------------- TMA producer
             uint32_t item_cnt = 0, it_cnt = 0;
@@ -309,21 +317,31 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: K-major x K-major
             constexpr uint32_t idesc_dv = make_idesc_bf16(128, D, 0, 1);    // A in TMEM / K-major smem, B MN-major
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 1, 1);    // A MN-major smem, B MN-major
-            const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v), ds_addr = smem_u32(sm.ds);
-            const uint32_t do_addr = smem_u32(sm.d_o);
-            const uint32_t ones_addr = smem_u32(&sm.ones[0][0]);
+            // Descriptors are built once; stepping along K only adds a byte offset (>> 4) to the
+            // start-address field, which cannot overflow for shared-memory addresses.
+            const uint64_t dk_k = make_desc_sw128(smem_u32(sm.k), 16, 1024);                   // K tile, K-major
+            const uint64_t dk_mn = make_desc_sw128(smem_u32(sm.k), Smem::kBoxBytes, 1024);     // K tile, MN-major
+            const uint64_t dv_k = make_desc_sw128(smem_u32(sm.v), 16, 1024);
+            const uint64_t ddo_k = make_desc_sw128(smem_u32(sm.d_o), 16, 1024);
+            const uint64_t ddo_mn = make_desc_sw128(smem_u32(sm.d_o), Smem::kBoxBytes, 1024);
+            const uint64_t dds_k = make_desc_sw128(smem_u32(sm.ds), 16, 1024);
+            const uint64_t dds_mn = make_desc_sw128(smem_u32(sm.ds), Smem::kBoxBytes, 1024);
+            const uint64_t dq_k0 = make_desc_sw128(smem_u32(sm.q[0]), 16, 1024);
+            const uint64_t dq_mn0 = make_desc_sw128(smem_u32(sm.q[0]), Smem::kBoxBytes, 1024);
+            const uint64_t daug0 = make_desc_noswizzle(smem_u32(sm.aug[0]), 2048, 128);
+            const uint64_t dones_s = make_desc_noswizzle(smem_u32(&sm.ones[1][0]), 2048, 128);  // ones, then zeros
+            const uint64_t dones_dp = make_desc_noswizzle(smem_u32(&sm.ones[0][0]), 2048, 128); // zeros, then ones
+            constexpr uint32_t kQStageStep = Smem::kTileBytes >> 4, kAugStageStep = 4096 >> 4;
             // S^T = K Q^T - LSE/scale: the last step multiplies the ones block with the LSE pieces
             auto issue_s = [&](uint32_t stage) {
                 ZL_PROF_SEG_BEGIN
-                const uint32_t q_addr = smem_u32(sm.q[stage]);
+                const uint64_t dq = dq_k0 + stage * kQStageStep;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                    mma_ss(tmem + kColS, make_desc_sw128(k_addr + off, 16, 1024),
-                           make_desc_sw128(q_addr + off, 16, 1024), idesc_s, ks > 0);
+                    const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
+                    mma_ss(tmem + kColS, dk_k + off, dq + off, idesc_s, ks > 0);
                 }
-                mma_ss(tmem + kColS, make_desc_noswizzle(ones_addr + 2048, 2048, 128),
-                       make_desc_noswizzle(smem_u32(sm.aug[stage]), 2048, 128), idesc_s, true);
+                mma_ss(tmem + kColS, dones_s, daug0 + stage * kAugStageStep, idesc_s, true);
                 mma_commit(&sm.s_full);
                 ZL_PROF_SEG_END(40)
             };
@@ -332,12 +350,10 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                    mma_ss(tmem + kColDP, make_desc_sw128(v_addr + off, 16, 1024),
-                           make_desc_sw128(do_addr + off, 16, 1024), idesc_s, ks > 0);
+                    const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
+                    mma_ss(tmem + kColDP, dv_k + off, ddo_k + off, idesc_s, ks > 0);
                 }
-                mma_ss(tmem + kColDP, make_desc_noswizzle(ones_addr, 2048, 128),
-                       make_desc_noswizzle(smem_u32(sm.aug[stage]), 2048, 128), idesc_s, true);
+                mma_ss(tmem + kColDP, dones_dp, daug0 + stage * kAugStageStep, idesc_s, true);
                 mma_commit(&sm.dp_full);
                 ZL_PROF_SEG_END(41)
             };
@@ -345,8 +361,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
-                    mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8,
-                           make_desc_sw128(do_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, acc || ks > 0);
+                    mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8, ddo_mn + ks * (2048 >> 4), idesc_dv,
+                           acc || ks > 0);
                 mma_commit(&sm.do_empty);
                 ZL_PROF_SEG_END(42)
             };
@@ -375,39 +391,48 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     issue_s(n1 & 1);  // overwrites P^T: ordered after dV on the tensor pipe
                 }
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
-                    const uint32_t q_addr = smem_u32(sm.q[it_cnt & 1]);
+                    const uint64_t dq_mn = dq_mn0 + (it_cnt & 1) * kQStageStep;
+                    ZL_TRACE(0, 0, it_cnt)
                     ZL_WAIT(&sm.ds_full, it_cnt & 1, 17);
+                    ZL_TRACE(0, 1, it_cnt)
                     tc_fence_after();
                     {
                         ZL_PROF_SEG_BEGIN
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
-                            mma_ss(tmem + kColDP, make_desc_sw128(ds_addr + ks * 2048, Smem::kBoxBytes, 1024),
-                                   make_desc_sw128(k_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dq, ks > 0);
+                            mma_ss(tmem + kColDP, dds_mn + ks * (2048 >> 4), dk_mn + ks * (2048 >> 4), idesc_dq, ks > 0);
                         mma_commit(&sm.dq_full);
+                        ZL_TRACE(0, 2, it_cnt)
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
-                            const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                            mma_ss(tmem + kColDK, make_desc_sw128(ds_addr + off, 16, 1024),
-                                   make_desc_sw128(q_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_dv, i > 0 || ks > 0);
+                            const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
+                            mma_ss(tmem + kColDK, dds_k + off, dq_mn + ks * (2048 >> 4), idesc_dv, i > 0 || ks > 0);
                         }
                         mma_commit(&sm.q_empty[it_cnt & 1]);
                         mma_commit(&sm.ds_free);
                         ZL_PROF_SEG_END(43)
                     }
+                    ZL_TRACE(0, 3, it_cnt)
                     if (i + 1 < n_it) {
                         const uint32_t n1 = it_cnt + 1, n2 = it_cnt + 2;
                         ZL_WAIT(&sm.do_full, n1 & 1, 18);
+                        ZL_TRACE(0, 4, it_cnt)
                         ZL_WAIT(&sm.dq_empty, it_cnt & 1, 19);
+                        ZL_TRACE(0, 5, it_cnt)
                         tc_fence_after();
                         issue_dp(n1 & 1);
+                        ZL_TRACE(0, 6, it_cnt)
                         ZL_WAIT(&sm.p_full, n1 & 1, 20);
+                        ZL_TRACE(0, 7, it_cnt)
                         tc_fence_after();
                         issue_dv(true);
+                        ZL_TRACE(0, 8, it_cnt)
                         if (i + 2 < n_it) {
                             ZL_WAIT(&sm.q_full[n2 & 1], (n2 >> 1) & 1, 16);
+                            ZL_TRACE(0, 9, it_cnt)
                             tc_fence_after();
                             issue_s(n2 & 1);
+                            ZL_TRACE(0, 10, it_cnt)
                         }
                     }
                 }
@@ -435,65 +460,96 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
                     const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
-                    const bool full = row_ok && q_valid == kTileQ;
+                    const bool tile_full = (wi.rows == kTileKV) && (q_valid == kTileQ);  // warp-uniform
+                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 0, it_cnt) }
                     ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 22);
+                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 1, it_cnt) }
                     tc_fence_after();
+                    ZL_PROF_SEG_BEGIN
                     uint32_t pk[32];  // P^T of this thread's row, bf16 pairs
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t sr[32];
-                        tmem_ld_x32(lane_addr + kColS + col0 + c * 32, sr);
+                    {
+                        uint32_t sr[2][32];
+                        tmem_ld_x32(lane_addr + kColS + col0, sr[0]);
+                        tmem_ld_x32(lane_addr + kColS + col0 + 32, sr[1]);
                         tmem_wait_ld();
-                        uint32_t pp[16];
+                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 6, it_cnt) }
+                        ZL_PROF_MARK(46)
+                        if (tile_full) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
-                            const int col = col0 + c * 32 + i;
-                            float p0 = ex2(__uint_as_float(sr[i]) * sl2);      // S^T already has -LSE/scale folded in
-                            float p1 = ex2(__uint_as_float(sr[i + 1]) * sl2);
-                            if (!full) {
-                                p0 = (row_ok && col < q_valid) ? p0 : 0.f;
-                                p1 = (row_ok && col + 1 < q_valid) ? p1 : 0.f;
+                            for (int c = 0; c < 2; ++c)
+#pragma unroll
+                                for (int i = 0; i < 32; i += 2)  // S^T already has -LSE/scale folded in
+                                    pk[c * 16 + i / 2] = pack_bf16(ex2(__uint_as_float(sr[c][i]) * sl2),
+                                                                   ex2(__uint_as_float(sr[c][i + 1]) * sl2));
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 2; ++c) {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 2) {
+                                    const int col = col0 + c * 32 + i;
+                                    float p0 = ex2(__uint_as_float(sr[c][i]) * sl2);
+                                    float p1 = ex2(__uint_as_float(sr[c][i + 1]) * sl2);
+                                    p0 = (row_ok && col < q_valid) ? p0 : 0.f;  // select, never multiply
+                                    p1 = (row_ok && col + 1 < q_valid) ? p1 : 0.f;
+                                    pk[c * 16 + i / 2] = pack_bf16(p0, p1);
+                                }
                             }
-                            pp[i / 2] = pack_bf16(p0, p1);
-                            pk[c * 16 + i / 2] = pp[i / 2];
                         }
-                        tmem_st_x16(lane_addr + kColS + col0 + c * 16, pp);
+                        ZL_PROF_MARK(47)
+                        tmem_st_x32(lane_addr + kColS + col0, pk);
+                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 7, it_cnt) }
                     }
                     tmem_wait_st();
+                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 8, it_cnt) }
                     tc_fence_before();
                     mbar_arrive(&sm.p_full);
+                    if (warp == 4 && lane == 0) { ZL_PROF_SEG_END(44) ZL_TRACE(1, 2, it_cnt) }
 
                     ZL_WAIT_WARP(&sm.dp_full, it_cnt & 1, 23);
+                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 3, it_cnt) }
                     if (it_cnt > 0) ZL_WAIT_WARP(&sm.ds_free, (it_cnt - 1) & 1, 24);  // dS buffer consumed by dK/dQ
+                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 4, it_cnt) }
                     tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t dr[32];
-                        tmem_ld_x32(lane_addr + kColDP + col0 + c * 32, dr);
+                    {
+                        ZL_PROF_SEG_BEGIN
+                        uint32_t dr[2][32];
+                        tmem_ld_x32(lane_addr + kColDP + col0, dr[0]);
+                        tmem_ld_x32(lane_addr + kColDP + col0 + 32, dr[1]);
                         tmem_wait_ld();
-                        uint32_t dd[16];
+                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 9, it_cnt) }
+                        ZL_PROF_MARK(48)
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
-                            const int col = col0 + c * 32 + i;
-                            const uint32_t pw = pk[c * 16 + i / 2];
-                            float d0 = __uint_as_float(pw << 16) * __uint_as_float(dr[i]);           // dP^T already has -D
-                            float d1 = __uint_as_float(pw & 0xffff0000u) * __uint_as_float(dr[i + 1]);
-                            if (!full) {
-                                d0 = (row_ok && col < q_valid) ? d0 : 0.f;
-                                d1 = (row_ok && col + 1 < q_valid) ? d1 : 0.f;
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t dd[16];
+                            if (tile_full) {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 2)  // dS^T = P^T o (dP^T - D) in packed bf16 arithmetic
+                                    dd[i / 2] = mul_bf16x2(pk[c * 16 + i / 2],
+                                                           pack_bf16(__uint_as_float(dr[c][i]), __uint_as_float(dr[c][i + 1])));
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 2) {
+                                    const int col = col0 + c * 32 + i;
+                                    float d0 = __uint_as_float(dr[c][i]), d1 = __uint_as_float(dr[c][i + 1]);
+                                    d0 = (row_ok && col < q_valid) ? d0 : 0.f;  // P is already zero there; keep 0 * garbage out
+                                    d1 = (row_ok && col + 1 < q_valid) ? d1 : 0.f;
+                                    dd[i / 2] = mul_bf16x2(pk[c * 16 + i / 2], pack_bf16(d0, d1));
+                                }
                             }
-                            dd[i / 2] = pack_bf16(d0, d1);
-                        }
 #pragma unroll
-                        for (int k4 = 0; k4 < 4; ++k4) {
-                            const int c16 = (col0 >> 3) + c * 4 + k4;  // 16-byte chunk index along the query axis
-                            const uint32_t addr = ds_row_addr + (c16 >> 3) * Smem::kBoxBytes + (((c16 & 7) ^ (row & 7)) << 4);
-                            st_shared_v4(addr, dd[k4 * 4], dd[k4 * 4 + 1], dd[k4 * 4 + 2], dd[k4 * 4 + 3]);
+                            for (int k4 = 0; k4 < 4; ++k4) {
+                                const int c16 = (col0 >> 3) + c * 4 + k4;  // 16-byte chunk index along the query axis
+                                const uint32_t addr = ds_row_addr + (c16 >> 3) * Smem::kBoxBytes + (((c16 & 7) ^ (row & 7)) << 4);
+                                st_shared_v4(addr, dd[k4 * 4], dd[k4 * 4 + 1], dd[k4 * 4 + 2], dd[k4 * 4 + 3]);
+                            }
                         }
+                        ZL_PROF_MARK(49)
+                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 10, it_cnt) }
+                        tc_fence_before();
+                        fence_proxy_async_smem();
+                        mbar_arrive(&sm.ds_full);
+                        if (warp == 4 && lane == 0) { ZL_PROF_SEG_END(45) ZL_TRACE(1, 5, it_cnt) }
                     }
-                    tc_fence_before();
-                    fence_proxy_async_smem();
-                    mbar_arrive(&sm.ds_full);
                 }
             }
             // ---- epilogue: warpgroup 0 stores dV, warpgroup 1 stores dK (scaled)
@@ -524,7 +580,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
     } else {
         // ------------------------------------------------------------------ dQ warpgroup (one query row per thread)
-        reg_inc<176>();
+        reg_inc<152>();
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
@@ -537,7 +593,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                 const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
+                    if (warp == 12 && lane == 0) { ZL_TRACE(2, 0, it_cnt) }
                     ZL_WAIT_WARP(&sm.dq_full, it_cnt & 1, 31);
+                    if (warp == 12 && lane == 0) { ZL_TRACE(2, 1, it_cnt) }
                     tc_fence_after();
                     if (p.dq_mode == 0) {
                         // vector reductions straight from registers
@@ -573,6 +631,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         tmem_wait_ld();
                         tc_fence_before();
                         mbar_arrive(&sm.dq_empty);
+                        if (warp == 12 && lane == 0) { ZL_TRACE(2, 2, it_cnt) }
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c, ++chunk_cnt) {
                             uint8_t* buf = sm.dq_stage;
