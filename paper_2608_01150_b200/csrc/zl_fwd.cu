@@ -1,14 +1,20 @@
 // Forward kernel of the coalesced attention engine (sm_100a).
 //
-// One persistent launch walks a longest-first list of work items (task, head, query tile)
-// that spans whole sequences and context-parallel shard tasks alike (paper Section IV-D:
-// all whole sequences of a rank are packed into one block-diagonal attention call next to
-// the rank's shards, without mixing attention across sequences).  Per item:
-//   S = Q K^T on the tensor cores (tcgen05.mma, operands staged by TMA in 128B-swizzled
-//   shared memory, accumulator in TMEM), online softmax in registers with one thread per
-//   query row, P written back to TMEM as bf16, O += P V on the tensor cores.
-// Whole-sequence tasks store final bf16 O and fp32 LSE; shard tasks store their partial
-// result (normalised within their own K/V chunk) as fp32 O plus LSE for the merge kernel.
+// One persistent launch walks a longest-first list of work items (task, head, 256-row query
+// block) that spans whole sequences and context-parallel shard tasks alike (paper Section
+// IV-D: all whole sequences of a rank are packed into one block-diagonal attention call next
+// to the rank's shards, without mixing attention across sequences).
+//
+// A CTA keeps TWO 128-row query tiles in flight so that the softmax of one overlaps the
+// tensor-core work of the other:
+//   warp 0      TMA producer: Q tiles once per item, K/V tiles through a shared-memory ring
+//   warp 1      MMA issuer:   S_x = Q_x K^T (tcgen05.mma, smem x smem -> TMEM) and
+//                             O_x += P_x V  (P read from TMEM, V from smem) for x in {A, B}
+//   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one thread per query row,
+//               online softmax with a lazily updated reference maximum, P written back over S
+//               in TMEM as bf16, final normalisation and stores.
+// Whole-sequence tasks store final bf16 O and fp32 LSE; shard tasks store their partial result
+// (normalised within their own K/V chunk) as fp32 O plus LSE for the merge kernel.
 #include <cuda_runtime.h>
 
 #include "zl_device.h"
@@ -20,8 +26,11 @@ using namespace ptx;
 
 namespace {
 
-constexpr int kFwdThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: softmax
+constexpr int kFwdThreads = 384;
 constexpr uint64_t kWaitLimitNs = 4000000000ull;
+// The reference maximum of a row is only raised when the tile maximum exceeds it by more than
+// this many powers of two; until then exponentials stay below 2^8 and nothing is rescaled.
+constexpr float kRescaleThresholdLog2 = 8.0f;
 
 template <int D>
 struct FwdSmem {
@@ -29,12 +38,12 @@ struct FwdSmem {
     static constexpr int kTileBytes = kTileQ * D * 2;  // one 128-row tile of Q, K or V
     static constexpr int kBoxBytes = kTileQ * 128;     // one TMA box: 128 rows x 64 bf16
     static constexpr int kBoxes = D / 64;
-    alignas(1024) uint8_t q[kTileBytes];
+    alignas(1024) uint8_t q[2][kTileBytes];
     alignas(1024) uint8_t k[kStages][kTileBytes];
     alignas(1024) uint8_t v[kStages][kTileBytes];
-    alignas(8) uint64_t q_full, q_empty;
-    uint64_t k_full[kStages], v_full[kStages], kv_empty[kStages];
-    uint64_t s_full, p_full, pv_done;
+    alignas(8) uint64_t q_full[2], q_empty;
+    uint64_t k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages];
+    uint64_t s_full[2], p_full[2], o_full[2];
     uint32_t tmem_base;
     volatile int32_t abort_flag;
 };
@@ -54,13 +63,13 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
     } while (0)
 // Wait used by all 32 lanes of a warp: the outcome is made warp-uniform and the warp
 // reconverges before the .sync.aligned TMEM instructions that follow.
-#define ZL_WAIT_WARP(bar, parity, site)                                             \
-    do {                                                                            \
+#define ZL_WAIT_WARP(bar, parity, site)                                              \
+    do {                                                                             \
         const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs) && !sm.abort_flag; \
-        if (!__all_sync(0xffffffffu, ok_)) {                                        \
-            report(p.status, &sm.abort_flag, 1000 + (site));                        \
-            goto teardown;                                                          \
-        }                                                                           \
+        if (!__all_sync(0xffffffffu, ok_)) {                                         \
+            report(p.status, &sm.abort_flag, 1000 + (site));                         \
+            goto teardown;                                                           \
+        }                                                                            \
     } while (0)
 
 template <int D>
@@ -70,26 +79,35 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     using Smem = FwdSmem<D>;
     constexpr int kStages = Smem::kStages;
     constexpr int kBoxes = Smem::kBoxes;
-    extern __shared__ uint8_t smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    // TMEM columns: S [0,128), O [128,128+D), P (bf16 pairs) [256,320)
-    constexpr uint32_t kColS = 0, kColO = 128, kColP = 256, kTmemCols = 512;
+    // TMEM columns: S_A [0,128), S_B [128,256), O_A [256,256+D), O_B [384,384+D).  P_x (bf16
+    // pairs) overwrites the first 64 columns of S_x once the row has been read.
+    constexpr uint32_t kColS = 0, kColO = 256, kTmemCols = 512;
 
+    if ((smem_u32(smem_raw) & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
+        if (threadIdx.x == 0 && atomicCAS(p.status, 0, (int)ZL_ERR_CUDA) == 0) p.status[1] = 1999;
+        return;
+    }
     if (threadIdx.x == 0) {
-        mbar_init(&sm.q_full, 1);
+        mbar_init(&sm.q_full[0], 1);
+        mbar_init(&sm.q_full[1], 1);
         mbar_init(&sm.q_empty, 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&sm.k_full[s], 1);
             mbar_init(&sm.v_full[s], 1);
-            mbar_init(&sm.kv_empty[s], 1);
+            mbar_init(&sm.k_empty[s], 1);
+            mbar_init(&sm.v_empty[s], 1);
         }
-        mbar_init(&sm.s_full, 1);
-        mbar_init(&sm.p_full, 128);
-        mbar_init(&sm.pv_done, 1);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&sm.s_full[x], 1);
+            mbar_init(&sm.p_full[x], 128);
+            mbar_init(&sm.o_full[x], 1);
+        }
         sm.abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tm_q);
@@ -105,179 +123,215 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t q_cnt = 0, kv_cnt = 0;
+    if (warp < 4) {
+        reg_dec<72>();
+        if (warp == 0 && lane == 0) {
+            // -------------------------------------------------------------- TMA producer
+            uint32_t q_cnt = 0, qb_cnt = 0, kv_cnt = 0;
             for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
                 const WorkItem wi = p.items[it];
                 const Task t = p.tasks[wi.unit];
                 const int n_kv = (t.kv_len + kTileKV - 1) / kTileKV;
                 if (n_kv == 0) continue;
+                const bool has_b = wi.rows > kTileQ;
                 ZL_WAIT(&sm.q_empty, (q_cnt & 1) ^ 1, 1);
-                mbar_arrive_expect_tx(&sm.q_full, Smem::kTileBytes);
-                for (int b = 0; b < kBoxes; ++b)
-                    tma_load_3d(sm.q + b * Smem::kBoxBytes, &tm_q, &sm.q_full, b * 64, wi.head, t.q_off + wi.row0);
                 ++q_cnt;
+                mbar_arrive_expect_tx(&sm.q_full[0], Smem::kTileBytes);
+                for (int b = 0; b < kBoxes; ++b)
+                    tma_load_3d(sm.q[0] + b * Smem::kBoxBytes, &tm_q, &sm.q_full[0], b * 64, wi.head, t.q_off + wi.row0);
                 for (int j = 0; j < n_kv; ++j, ++kv_cnt) {
                     const int s = kv_cnt % kStages;
                     const uint32_t ph = (kv_cnt / kStages) & 1;
-                    ZL_WAIT(&sm.kv_empty[s], ph ^ 1, 2);
+                    ZL_WAIT(&sm.k_empty[s], ph ^ 1, 2);
                     mbar_arrive_expect_tx(&sm.k_full[s], Smem::kTileBytes);
                     for (int b = 0; b < kBoxes; ++b)
                         tma_load_3d(sm.k[s] + b * Smem::kBoxBytes, &tm_k, &sm.k_full[s], b * 64, wi.head,
                                     t.kv_off + j * kTileKV);
+                    if (j == 0 && has_b) {  // second query tile right after the first K tile
+                        mbar_arrive_expect_tx(&sm.q_full[1], Smem::kTileBytes);
+                        for (int b = 0; b < kBoxes; ++b)
+                            tma_load_3d(sm.q[1] + b * Smem::kBoxBytes, &tm_q, &sm.q_full[1], b * 64, wi.head,
+                                        t.q_off + wi.row0 + kTileQ);
+                        ++qb_cnt;
+                    }
+                    ZL_WAIT(&sm.v_empty[s], ph ^ 1, 3);
                     mbar_arrive_expect_tx(&sm.v_full[s], Smem::kTileBytes);
                     for (int b = 0; b < kBoxes; ++b)
                         tma_load_3d(sm.v[s] + b * Smem::kBoxBytes, &tm_v, &sm.v_full[s], b * 64, wi.head,
                                     t.kv_off + j * kTileKV);
                 }
             }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        } else if (warp == 1 && lane == 0) {
+            // -------------------------------------------------------------- MMA issuer
             constexpr uint32_t idesc_s = make_idesc_bf16(kTileQ, kTileKV, 0, 0);
             constexpr uint32_t idesc_o = make_idesc_bf16(kTileQ, D, 0, 1);
-            uint32_t q_cnt = 0, kv_cnt = 0, p_cnt = 0;
-            const uint32_t q_addr = smem_u32(sm.q);
+            const uint64_t dq0 = make_desc_sw128(smem_u32(sm.q[0]), 16, 1024);
+            const uint64_t dk0 = make_desc_sw128(smem_u32(sm.k[0]), 16, 1024);
+            const uint64_t dv0 = make_desc_sw128(smem_u32(sm.v[0]), Smem::kBoxBytes, 1024);  // V is the MN-major B operand
+            constexpr uint32_t kTileStep = Smem::kTileBytes >> 4;
+            // S_x = Q_x K^T
+            auto issue_s = [&](int x, uint32_t stage) {
+                const uint64_t dq = dq0 + x * kTileStep, dk = dk0 + stage * kTileStep;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
+                    mma_ss(tmem + kColS + x * 128, dq + off, dk + off, idesc_s, ks > 0);
+                }
+                mma_commit(&sm.s_full[x]);
+            };
+            // O_x (+)= P_x V
+            auto issue_pv = [&](int x, uint32_t stage, bool acc) {
+                const uint64_t dv = dv0 + stage * kTileStep;
+#pragma unroll
+                for (int ks = 0; ks < kTileKV / 16; ++ks)
+                    mma_ts(tmem + kColO + x * 128, tmem + kColS + x * 128 + ks * 8, dv + ks * (2048 >> 4), idesc_o,
+                           acc || ks > 0);
+            };
+            uint32_t q_cnt = 0, qb_cnt = 0, kv_cnt = 0, pa_cnt = 0, pb_cnt = 0;
             for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
                 const WorkItem wi = p.items[it];
                 const Task t = p.tasks[wi.unit];
                 const int n_kv = (t.kv_len + kTileKV - 1) / kTileKV;
                 if (n_kv == 0) continue;
-                ZL_WAIT(&sm.q_full, q_cnt & 1, 11);
+                const bool has_b = wi.rows > kTileQ;
+                ZL_WAIT(&sm.q_full[0], q_cnt & 1, 11);
                 ++q_cnt;
-                auto issue_s = [&](uint32_t stage) {
-                    const uint32_t k_addr = smem_u32(sm.k[stage]);
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t off = (ks / 4) * Smem::kBoxBytes + (ks % 4) * 32;
-                        mma_ss(tmem + kColS, make_desc_sw128(q_addr + off, 16, 1024),
-                               make_desc_sw128(k_addr + off, 16, 1024), idesc_s, ks > 0);
-                    }
-                    mma_commit(&sm.s_full);
-                };
                 ZL_WAIT(&sm.k_full[kv_cnt % kStages], (kv_cnt / kStages) & 1, 12);
-                issue_s(kv_cnt % kStages);
+                tc_fence_after();
+                issue_s(0, kv_cnt % kStages);
+                if (has_b) {
+                    ZL_WAIT(&sm.q_full[1], qb_cnt & 1, 13);
+                    ++qb_cnt;
+                    tc_fence_after();
+                    issue_s(1, kv_cnt % kStages);
+                }
+                mma_commit(&sm.k_empty[kv_cnt % kStages]);
+                if (n_kv == 1) mma_commit(&sm.q_empty);
                 for (int j = 0; j < n_kv; ++j, ++kv_cnt) {
-                    const uint32_t s = kv_cnt % kStages;
-                    // P(j) written, S(j) fully read, O rescaled
-                    ZL_WAIT(&sm.p_full, p_cnt & 1, 13);
-                    ++p_cnt;
-                    if (j + 1 < n_kv) {
-                        const uint32_t nk = kv_cnt + 1;
-                        ZL_WAIT(&sm.k_full[nk % kStages], (nk / kStages) & 1, 14);
-                        issue_s(nk % kStages);
-                    } else {
-                        mma_commit(&sm.q_empty);  // all S MMAs of this item are done with Q
-                    }
+                    const uint32_t s = kv_cnt % kStages, nk = kv_cnt + 1, sn = nk % kStages;
+                    const bool has_next = j + 1 < n_kv;
+                    // tile A: P_A(j) is in TMEM (S_A(j) fully read, O_A rescaled if needed)
+                    ZL_WAIT(&sm.p_full[0], pa_cnt & 1, 14);
+                    ++pa_cnt;
                     ZL_WAIT(&sm.v_full[s], (kv_cnt / kStages) & 1, 15);
                     tc_fence_after();
-                    const uint32_t v_addr = smem_u32(sm.v[s]);
-#pragma unroll
-                    for (int ks = 0; ks < kTileKV / 16; ++ks) {
-                        mma_ts(tmem + kColO, tmem + kColP + ks * 8,
-                               make_desc_sw128(v_addr + ks * 2048, Smem::kBoxBytes, 1024), idesc_o,
-                               j > 0 || ks > 0);
+                    issue_pv(0, s, j > 0);
+                    if (!has_next) mma_commit(&sm.o_full[0]);
+                    if (has_next) {
+                        ZL_WAIT(&sm.k_full[sn], (nk / kStages) & 1, 16);
+                        tc_fence_after();
+                        issue_s(0, sn);  // overwrites P_A(j): ordered after P_A V on the tensor pipe
                     }
-                    mma_commit(&sm.kv_empty[s]);
-                    mma_commit(&sm.pv_done);
+                    if (has_b) {
+                        ZL_WAIT(&sm.p_full[1], pb_cnt & 1, 17);
+                        ++pb_cnt;
+                        tc_fence_after();
+                        issue_pv(1, s, j > 0);
+                        if (!has_next) mma_commit(&sm.o_full[1]);
+                    }
+                    mma_commit(&sm.v_empty[s]);
+                    if (has_next) {
+                        if (has_b) issue_s(1, sn);
+                        mma_commit(&sm.k_empty[sn]);
+                        if (j + 2 == n_kv) mma_commit(&sm.q_empty);  // last S of the item issued
+                    }
                 }
             }
         }
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
+        reg_inc<216>();
+        const int x = (warp - 4) >> 2;             // 0: tile A, 1: tile B
         const int quarter = warp & 3;              // TMEM lane quarter this warp may access
         const int row = quarter * 32 + lane;       // query row within the tile
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-        uint32_t s_cnt = 0, pv_cnt = 0;
+        const uint32_t col_s = kColS + x * 128, col_o = kColO + x * 128;
+        uint32_t s_cnt = 0, o_cnt = 0;
         const float sl2 = p.scale_log2;
         for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
             const WorkItem wi = p.items[it];
+            const int tile_rows = min(kTileQ, wi.rows - x * kTileQ);  // rows of this warpgroup's tile
+            if (tile_rows <= 0) continue;
             const Task t = p.tasks[wi.unit];
             const int n_kv = (t.kv_len + kTileKV - 1) / kTileKV;
-            float m = -INFINITY, l = 0.f;
+            float m_ref = -INFINITY, l = 0.f;  // reference maximum (raw score units) and row sum
             for (int j = 0; j < n_kv; ++j) {
-                ZL_WAIT_WARP(&sm.s_full, s_cnt & 1, 21);
+                ZL_WAIT_WARP(&sm.s_full[x], s_cnt & 1, 21);
                 ++s_cnt;
                 tc_fence_after();
                 float sv[kTileKV];
 #pragma unroll
                 for (int c = 0; c < kTileKV / 32; ++c) {
                     uint32_t r[32];
-                    tmem_ld_x32(lane_addr + kColS + c * 32, r);
-                    tmem_wait_ld();
+                    tmem_ld_x32(lane_addr + col_s + c * 32, r);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) sv[c * 32 + i] = __uint_as_float(r[i]);
                 }
+                tmem_wait_ld();
                 const int valid = t.kv_len - j * kTileKV;  // columns of this tile inside the task
                 if (valid < kTileKV) {
 #pragma unroll
                     for (int c = 0; c < kTileKV; ++c)
-                        if (c >= valid) sv[c] = -INFINITY;
+                        if (c >= valid) sv[c] = -INFINITY;  // select, never multiply
                 }
-                float mx = sv[0];
+                float mx = max3(sv[0], sv[1], sv[2]);
 #pragma unroll
-                for (int c = 1; c < kTileKV; ++c) mx = fmaxf(mx, sv[c]);
-                const float m_new = fmaxf(m, mx);
-                const float alpha = ex2((m - m_new) * sl2);
-                const float mb = m_new * sl2;
-                float rs = 0.f;
-                uint32_t pk[kTileKV / 2];
-#pragma unroll
-                for (int c = 0; c < kTileKV; c += 2) {
-                    const float p0 = ex2(fmaf(sv[c], sl2, -mb));
-                    const float p1 = ex2(fmaf(sv[c + 1], sl2, -mb));
-                    rs += p0 + p1;
-                    pk[c / 2] = pack_bf16(p0, p1);
-                }
-                l = l * alpha + rs;
-                m = m_new;
-                if (j > 0) {
-                    // previous P V product must be complete before O is rescaled and P overwritten
-                    ZL_WAIT_WARP(&sm.pv_done, pv_cnt & 1, 22);
-                    ++pv_cnt;
-                    tc_fence_after();
+                for (int c = 3; c + 1 < kTileKV; c += 2) mx = max3(mx, sv[c], sv[c + 1]);
+                mx = fmaxf(mx, sv[kTileKV - 1]);
+                // lazy reference update: only when the tile maximum is far above the reference
+                const bool raise = (mx - m_ref) * sl2 > kRescaleThresholdLog2;
+                if (__any_sync(0xffffffffu, raise && j > 0)) {
+                    // rescale O (the previous P V product is complete: S(j) was issued after it)
+                    const float alpha = raise ? ex2((m_ref - mx) * sl2) : 1.f;
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
-                        tmem_ld_x32(lane_addr + kColO + c * 32, r);
+                        tmem_ld_x32(lane_addr + col_o + c * 32, r);
                         tmem_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st_x32(lane_addr + kColO + c * 32, r);
+                        tmem_st_x32(lane_addr + col_o + c * 32, r);
                     }
+                    l *= alpha;
                 }
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t r[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = pk[c * 32 + i];
-                    tmem_st_x32(lane_addr + kColP + c * 32, r);
+                if (raise) {
+                    if (j == 0) l = 0.f;
+                    m_ref = mx;
                 }
+                const float nmb = -m_ref * sl2;
+                float2 sum2 = make_float2(0.f, 0.f);
+                uint32_t pk[kTileKV / 2];
+#pragma unroll
+                for (int c = 0; c < kTileKV; c += 2) {
+                    const float2 e = fma2(make_float2(sv[c], sv[c + 1]), make_float2(sl2, sl2), make_float2(nmb, nmb));
+                    const float p0 = ex2(e.x), p1 = ex2(e.y);
+                    sum2 = add2(sum2, make_float2(p0, p1));
+                    pk[c / 2] = pack_bf16(p0, p1);
+                }
+                l += sum2.x + sum2.y;
+                tmem_st_x32(lane_addr + col_s, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+                tmem_st_x32(lane_addr + col_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(&sm.p_full);
+                mbar_arrive(&sm.p_full[x]);
             }
             // ---- epilogue
-            const bool row_ok = row < wi.rows;
+            const bool row_ok = row < tile_rows;
             const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
-            const float lse = (l > 0.f) ? (m * sl2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            const float lse = (l > 0.f) ? (m_ref * sl2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
             if (n_kv > 0) {
-                ZL_WAIT_WARP(&sm.pv_done, pv_cnt & 1, 23);
-                ++pv_cnt;
+                ZL_WAIT_WARP(&sm.o_full[x], o_cnt & 1, 23);
+                ++o_cnt;
                 tc_fence_after();
             }
-            const int64_t grow = (int64_t)(t.partial_slot >= 0 ? t.partial_slot : t.q_off) + wi.row0 + row;
+            const int64_t grow = (int64_t)(t.partial_slot >= 0 ? t.partial_slot : t.q_off) + wi.row0 + x * kTileQ + row;
             if (t.partial_slot >= 0) {
                 float* dst = p.o_partial + (grow * p.n_heads + wi.head) * D;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t r[32];
                     if (n_kv > 0) {
-                        tmem_ld_x32(lane_addr + kColO + c * 32, r);
+                        tmem_ld_x32(lane_addr + col_o + c * 32, r);
                         tmem_wait_ld();
                     } else {
 #pragma unroll
@@ -299,7 +353,7 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t r[32];
                     if (n_kv > 0) {
-                        tmem_ld_x32(lane_addr + kColO + c * 32, r);
+                        tmem_ld_x32(lane_addr + col_o + c * 32, r);
                         tmem_wait_ld();
                     } else {
 #pragma unroll
@@ -333,31 +387,26 @@ teardown:
     }
 }
 
+template <int D>
+cudaError_t launch_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                     int grid, cudaStream_t stream) {
+    constexpr int smem = sizeof(FwdSmem<D>);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(zl_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    zl_fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, p);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                        const FwdParams& p, int grid, cudaStream_t stream) {
     if (p.n_items == 0) return cudaSuccess;
-    if (head_dim == 128) {
-        constexpr int smem = sizeof(FwdSmem<128>) + 1024;
-        static bool configured = false;
-        if (!configured) {
-            cudaError_t e = cudaFuncSetAttribute(zl_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            if (e != cudaSuccess) return e;
-            configured = true;
-        }
-        zl_fwd_kernel<128><<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, p);
-    } else {
-        constexpr int smem = sizeof(FwdSmem<64>) + 1024;
-        static bool configured = false;
-        if (!configured) {
-            cudaError_t e = cudaFuncSetAttribute(zl_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            if (e != cudaSuccess) return e;
-            configured = true;
-        }
-        zl_fwd_kernel<64><<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, p);
-    }
-    return cudaGetLastError();
+    return head_dim == 128 ? launch_t<128>(tq, tk, tv, p, grid, stream) : launch_t<64>(tq, tk, tv, p, grid, stream);
 }
 
 }  // namespace zl

@@ -10,7 +10,7 @@ namespace zl {
 
 constexpr int kTileQ = 128;   // query rows per MMA tile (TMEM lanes)
 constexpr int kTileKV = 128;  // key rows per MMA tile
-constexpr int kFwdBlockQ = kTileQ;  // query rows per forward work item
+constexpr int kFwdBlockQ = 2 * kTileQ;  // query rows per forward work item: two tiles in flight per CTA
 
 // One attention task on the device: whole sequence or shard.
 struct alignas(32) Task {
