@@ -49,37 +49,60 @@ int orc_num_threads(void) {
 #endif
 }
 
+/* Query rows are processed in groups of ORC_GROUP rows that share each pass over the keys
+ * (so a long key set is streamed from memory once per group instead of once per row); the
+ * arithmetic of every row, and the order of its sums, is exactly the one written above. */
+#define ORC_GROUP 8
+
 /* Forward for query rows listed in `rows` (NULL: rows 0..n_rows-1).  Output r belongs to
  * query row rows[r]; O has n_rows rows with stride ldo, lse has n_rows entries. */
 void orc_attn_fwd(const double* q, long ldq, const double* k, long ldk, const double* v, long ldv,
                   long n_kv, int d, double scale, const long* rows, long n_rows,
                   double* O, long ldo, double* lse) {
+    const long n_groups = (n_rows + ORC_GROUP - 1) / ORC_GROUP;
 #pragma omp parallel
     {
-        double* s = (double*)malloc(sizeof(double) * (size_t)(n_kv > 0 ? n_kv : 1));
-#pragma omp for schedule(dynamic, 4)
-        for (long r = 0; r < n_rows; ++r) {
-            const long i = rows ? rows[r] : r;
-            const double* qi = q + i * ldq;
-            double* Oi = O + r * ldo;
-            for (int c = 0; c < d; ++c) Oi[c] = 0.0;
-            if (n_kv <= 0) { lse[r] = -INFINITY; continue; }
-            double m = -INFINITY;
-            for (long j = 0; j < n_kv; ++j) {
-                const double* kj = k + j * ldk;
-                double acc = 0.0;
-                for (int c = 0; c < d; ++c) acc += qi[c] * kj[c];
-                s[j] = scale * acc;
-                if (s[j] > m) m = s[j];
+        double* s = (double*)malloc(sizeof(double) * (size_t)ORC_GROUP * (size_t)(n_kv > 0 ? n_kv : 1));
+#pragma omp for schedule(dynamic, 1)
+        for (long g = 0; g < n_groups; ++g) {
+            const long r0 = g * ORC_GROUP;
+            const int nr = (int)((n_rows - r0 < ORC_GROUP) ? (n_rows - r0) : ORC_GROUP);
+            const double* qi[ORC_GROUP];
+            double m[ORC_GROUP], L[ORC_GROUP];
+            for (int a = 0; a < nr; ++a) {
+                const long i = rows ? rows[r0 + a] : (r0 + a);
+                qi[a] = q + i * ldq;
+                double* Oi = O + (r0 + a) * ldo;
+                for (int c = 0; c < d; ++c) Oi[c] = 0.0;
+                m[a] = -INFINITY;
             }
-            double l = 0.0;
-            for (long j = 0; j < n_kv; ++j) l += exp(s[j] - m);
-            const double L = m + log(l);
-            lse[r] = L;
-            for (long j = 0; j < n_kv; ++j) {
-                const double p = exp(s[j] - L);
+            if (n_kv <= 0) {
+                for (int a = 0; a < nr; ++a) lse[r0 + a] = -INFINITY;
+                continue;
+            }
+            for (long j = 0; j < n_kv; ++j) {          /* scores and row maxima */
+                const double* kj = k + j * ldk;
+                for (int a = 0; a < nr; ++a) {
+                    double acc = 0.0;
+                    for (int c = 0; c < d; ++c) acc += qi[a][c] * kj[c];
+                    const double sj = scale * acc;
+                    s[(size_t)a * n_kv + j] = sj;
+                    if (sj > m[a]) m[a] = sj;
+                }
+            }
+            for (int a = 0; a < nr; ++a) {             /* log-sum-exp */
+                double l = 0.0;
+                for (long j = 0; j < n_kv; ++j) l += exp(s[(size_t)a * n_kv + j] - m[a]);
+                L[a] = m[a] + log(l);
+                lse[r0 + a] = L[a];
+            }
+            for (long j = 0; j < n_kv; ++j) {          /* O_i = sum_j p_ij v_j */
                 const double* vj = v + j * ldv;
-                for (int c = 0; c < d; ++c) Oi[c] += p * vj[c];
+                for (int a = 0; a < nr; ++a) {
+                    const double p = exp(s[(size_t)a * n_kv + j] - L[a]);
+                    double* Oi = O + (r0 + a) * ldo;
+                    for (int c = 0; c < d; ++c) Oi[c] += p * vj[c];
+                }
             }
         }
         free(s);
@@ -128,22 +151,32 @@ void orc_attn_bwd_dq(const double* q, long ldq, const double* k, long ldk, const
                      const double* dO, long lddo, const double* lse, const double* D,
                      long n_kv, int d, double scale, const long* rows, long n_rows,
                      double* dQ, long lddq) {
-#pragma omp parallel for schedule(dynamic, 4)
-    for (long r = 0; r < n_rows; ++r) {
-        const long i = rows ? rows[r] : r;
-        const double* qi = q + i * ldq;
-        const double* doi = dO + i * lddo;
-        double* dqi = dQ + r * lddq;
-        for (int c = 0; c < d; ++c) dqi[c] = 0.0;
+    const long n_groups = (n_rows + ORC_GROUP - 1) / ORC_GROUP;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long g = 0; g < n_groups; ++g) {
+        const long r0 = g * ORC_GROUP;
+        const int nr = (int)((n_rows - r0 < ORC_GROUP) ? (n_rows - r0) : ORC_GROUP);
+        long idx[ORC_GROUP];
+        for (int a = 0; a < nr; ++a) {
+            idx[a] = rows ? rows[r0 + a] : (r0 + a);
+            double* dqi = dQ + (r0 + a) * lddq;
+            for (int c = 0; c < d; ++c) dqi[c] = 0.0;
+        }
         if (n_kv <= 0) continue;
         for (long j = 0; j < n_kv; ++j) {
             const double* kj = k + j * ldk;
             const double* vj = v + j * ldv;
-            double s = 0.0, dp = 0.0;
-            for (int c = 0; c < d; ++c) { s += qi[c] * kj[c]; dp += doi[c] * vj[c]; }
-            const double p = exp(scale * s - lse[i]);
-            const double ds = p * (dp - D[i]);
-            for (int c = 0; c < d; ++c) dqi[c] += scale * ds * kj[c];
+            for (int a = 0; a < nr; ++a) {
+                const long i = idx[a];
+                const double* qi = q + i * ldq;
+                const double* doi = dO + i * lddo;
+                double* dqi = dQ + (r0 + a) * lddq;
+                double s = 0.0, dp = 0.0;
+                for (int c = 0; c < d; ++c) { s += qi[c] * kj[c]; dp += doi[c] * vj[c]; }
+                const double p = exp(scale * s - lse[i]);
+                const double ds = p * (dp - D[i]);
+                for (int c = 0; c < d; ++c) dqi[c] += scale * ds * kj[c];
+            }
         }
     }
 }

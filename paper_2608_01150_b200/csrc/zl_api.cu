@@ -370,10 +370,6 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     p.q_pad_total = (int32_t)s.q_pad_total;
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
-    {
-        const char* e = getenv("ZL_DQ_MODE");
-        p.dq_mode = e ? atoi(e) : 1;
-    }
     p.o = static_cast<const __nv_bfloat16*>(o);
     p.d_o = static_cast<const __nv_bfloat16*>(d_o);
     p.lse = lse;

@@ -16,7 +16,8 @@
 //         K, V in shared memory and dK, dV in TMEM, and loops over every 128-row query tile
 //         of every task that shares the key range.  Per tile it issues five tcgen05 MMAs
 //         (S^T = K Q^T, dP^T = V dO^T, dV += P^T dO, dK += dS^T Q, dQ = dS K); dK/dV need no
-//         atomics, dQ tiles are added into an fp32 accumulator with vector reductions;
+//         atomics, dQ tiles are staged in shared memory and added into an fp32 accumulator by
+//         the TMA (cp.reduce.async.bulk.tensor);
 //   post  dQ accumulator * scale -> bf16.
 #include <cuda_runtime.h>
 
@@ -597,27 +598,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ZL_WAIT_WARP(&sm.dq_full, it_cnt & 1, 31);
                     if (warp == 12 && lane == 0) { ZL_TRACE(2, 1, it_cnt) }
                     tc_fence_after();
-                    if (p.dq_mode == 0) {
-                        // vector reductions straight from registers
-                        const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
-                        float* dst = p.dq_acc + (((int64_t)t.q_slot + qt * kTileQ + row) * p.n_heads + wi.head) * D;
-#pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t r[32];
-                            tmem_ld_x32(lane_addr + kColDP + c * 32, r);
-                            tmem_wait_ld();
-                            if (c == D / 32 - 1) {
-                                tc_fence_before();
-                                mbar_arrive(&sm.dq_empty);
-                            }
-                            if (row < q_valid) {
-#pragma unroll
-                                for (int i = 0; i < 32; i += 4)
-                                    red_add_v4(dst + c * 32 + i, __uint_as_float(r[i]), __uint_as_float(r[i + 1]),
-                                               __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                            }
-                        }
-                    } else {
+                    {
                         // read the whole tile (frees the TMEM columns for the next dP^T), then stage
                         // 32-column chunks in swizzled shared memory and add them with the TMA
                         uint32_t r[D];

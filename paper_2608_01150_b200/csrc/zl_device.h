@@ -51,7 +51,6 @@ struct BwdParams {
     int32_t q_pad_total;
     float scale;
     float scale_log2;
-    int32_t dq_mode;  // 0: vector reductions from registers, 1: TMA reduce-add from shared memory
     const __nv_bfloat16* o;
     const __nv_bfloat16* d_o;
     const float* lse;
