@@ -107,6 +107,25 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------
+# multi-rank helpers (also exercised on CPU with gloo by tests/test_multirank_cpu.py)
+# --------------------------------------------------------------------------------------
+def reduce_max_ms(ms: float, dist, device) -> float:
+    """Slowest rank's time: every rank contributes its device-timed milliseconds."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tflops(world: int, flops_per_rank: float, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank runs its own rank-local placement of the same shape
+    (weak scaling, no data-path collective), so the job does world * flops in the slowest time."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
+# --------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------
 class Workload:
@@ -160,12 +179,9 @@ class Workload:
             fn()
         e1.record()
         torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
+        ms = reduce_max_ms(e0.elapsed_time(e1), dist, self.Q.device)
         if dist is not None:
-            t = torch.tensor([ms], dtype=torch.float64, device=self.Q.device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
             dist.barrier()
-            ms = float(t.item())
         return ms
 
     def make_host_buffers(self):
@@ -255,7 +271,7 @@ def run_ours(args):
     clocks = sampler.stop()
     ms_step = ms_total / K
     flops = p.fwd_flops() + p.bwd_flops()
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = aggregate_tflops(world, flops, ms_step)
 
     # per-kernel device time (separate pass with event brackets around every launch)
     wl.h.set_kernel_timing(True)
@@ -284,7 +300,7 @@ def run_ours(args):
     for _ in range(2):
         wl.e2e_step()
     ms_e2e = wl.time_region(wl.e2e_step, K, dist) / K
-    e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+    e2e = {"value": aggregate_tflops(world, flops, ms_e2e), "unit": "TFLOP/s", "ms_per_step": ms_e2e,
            "h2d_bytes_per_step": wl.h2d_bytes, "d2h_bytes_per_step": wl.d2h_bytes}
     code, where = wl.h.last_device_status()
     if code != 0:
@@ -299,7 +315,7 @@ def run_ours(args):
                    "step": "fwd launch + lse merge + bwd (pre, main, post)",
                    "l2": "inputs larger than L2 (K+V alone exceed 126 MB); no flush",
                    "parallelism": f"{world} independent rank-local placements"},
-        "fwd_tflops": world * p.fwd_flops() / (ms_fwd / K * 1e-3) / 1e12,
+        "fwd_tflops": aggregate_tflops(world, p.fwd_flops(), ms_fwd / K),
         "fwd_ms": ms_fwd / K,
         "frac_of_peak": {"burst_1645.7": value / world / float(peaks.get("bf16_tflops", 1590.0)),
                          "sustained": value / world / peak_t, "datasheet_2250": value / world / 2250.0},
