@@ -158,6 +158,36 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* tasks, const void* q, const void
                                 void* dq, void* dk, void* dv,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* zl_coalesced_attn_bwd_noalloc -- the backward for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a convenience of the library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a stream-ordered region
+ * owned by another allocator, in a plugin whose host forbids allocations after initialisation, or
+ * on a latency-critical path where an allocator call (and the implicit synchronisation it may
+ * bring) is not acceptable -- and that therefore has no workspace buffer to hand to
+ * zl_coalesced_attn_bwd.  This entry point takes the same inputs and outputs but no workspace:
+ * the scratch (fp32 dQ accumulator and the per-tile LSE/D tiles) lives in a fixed device array
+ * of ZL_NOALLOC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the
+ * library reserves that much memory until the process exits.
+ *
+ *   - Placements whose zl_tasks_info.bwd_workspace_bytes exceeds ZL_NOALLOC_SCRATCH_BYTES are
+ *     rejected with ZL_ERR_WORKSPACE; nothing is launched.
+ *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating routine.  The task
+ *     handle must have been built beforehand (zl_build_tasks allocates its small tables), and
+ *     kernel timing must be off on the handle (ZL_ERR_INVALID_ARG otherwise: timing creates events).
+ *   - The first call on each device looks up the device address of the scratch array; make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it.
+ *     The part that must start at zero (the dQ accumulator) is cleared on the stream by every
+ *     call.  Two calls that overlap on the GPU (different streams, or different handles at the
+ *     same time) race on the array and produce garbage: serialise them.
+ * Results equal those of zl_coalesced_attn_bwd (dK, dV bit for bit; dQ up to the order of the
+ * fp32 reduce-adds). */
+#define ZL_NOALLOC_SCRATCH_BYTES (64u * 1024u * 1024u)
+zl_status zl_coalesced_attn_bwd_noalloc(const zl_tasks* tasks, const void* q, const void* k, const void* v,
+                                        const void* o, const float* lse, const void* d_o, float scale,
+                                        void* dq, void* dk, void* dv, void* stream);
+
 /* Synchronises the handle's device and reads the device status word written by the
  * kernels: code is ZL_OK or ZL_ERR_TIMEOUT, `where` identifies the wait that expired
  * (kernel id * 1000 + site).  Resets the word to ZL_OK. */

@@ -6,5 +6,6 @@ kernels.  PyTorch is used for device memory and streams.  There is no CPU fallba
 ``libzellige.so`` has not been built, importing :mod:`.binding` raises.
 """
 from .binding import (ZlError, TaskHandle, ShardDesc, TasksInfo, build_tasks,  # noqa: F401
-                      coalesced_attn_fwd, lse_merge, coalesced_attn_bwd, launch_count,
+                      coalesced_attn_fwd, lse_merge, coalesced_attn_bwd, coalesced_attn_bwd_noalloc,
+                      NOALLOC_SCRATCH_BYTES, launch_count,
                       library_path, STATUS_NAMES)

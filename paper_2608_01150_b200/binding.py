@@ -69,6 +69,8 @@ def _load():
     lib.zl_coalesced_attn_bwd.restype = ctypes.c_int
     lib.zl_coalesced_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
+    lib.zl_coalesced_attn_bwd_noalloc.restype = ctypes.c_int
+    lib.zl_coalesced_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.zl_last_device_status.restype = ctypes.c_int
     lib.zl_last_device_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.zl_set_kernel_timing.restype = ctypes.c_int
@@ -209,6 +211,19 @@ def coalesced_attn_bwd(tasks: TaskHandle, q, k, v, o, lse, d_o, scale: float, dq
                                       ctypes.c_float(scale), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
                                       ctypes.c_size_t(workspace_bytes), _stream_ptr(stream)),
            "zl_coalesced_attn_bwd")
+
+
+NOALLOC_SCRATCH_BYTES = 64 * 1024 * 1024
+
+
+def coalesced_attn_bwd_noalloc(tasks: TaskHandle, q, k, v, o, lse, d_o, scale: float, dq, dk, dv, stream=None):
+    """zl_coalesced_attn_bwd_noalloc: the backward for callers that cannot allocate device memory
+    (no workspace argument; the scratch is a fixed 64 MiB array inside the library).  Raises
+    ZL_ERR_WORKSPACE for placements that need more scratch than that.  Calls must not overlap on
+    the GPU, and the first call on a device should be made outside stream capture."""
+    _check(_lib.zl_coalesced_attn_bwd_noalloc(tasks.ptr, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o),
+                                              ctypes.c_float(scale), _ptr(dq), _ptr(dk), _ptr(dv),
+                                              _stream_ptr(stream)), "zl_coalesced_attn_bwd_noalloc")
 
 
 def launch_count() -> int:

@@ -433,6 +433,46 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     return ZL_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Backward without a caller-provided workspace: the scratch is a fixed array in the library image.
+// In host code `g_noalloc_scratch` is only a handle for the symbol, not a device address; the
+// address is looked up once per device and cached.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[ZL_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (nullptr on failure).
+void* noalloc_scratch_for(int device) {
+    if (device < 0 || device >= kMaxDevices) return nullptr;
+    if (!g_noalloc_ptr[device]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        g_noalloc_ptr[device] = ptr;
+    }
+    return g_noalloc_ptr[device];
+}
+}  // namespace
+
+zl_status zl_coalesced_attn_bwd_noalloc(const zl_tasks* t, const void* q, const void* k, const void* v,
+                                        const void* o, const float* lse, const void* d_o, float scale, void* dq,
+                                        void* dk, void* dv, void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    if (t->sched.tasks.empty()) return ZL_OK;
+    if (t->device < 0) return ZL_ERR_CUDA;
+    if (t->timing) return ZL_ERR_INVALID_ARG;  // per-kernel timing creates events: not allocation-free
+    if (t->sched.bwd_workspace_bytes > (size_t)ZL_NOALLOC_SCRATCH_BYTES) return ZL_ERR_WORKSPACE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != t->device) return ZL_ERR_CUDA;
+    void* scratch = noalloc_scratch_for(dev);
+    if (!scratch) return ZL_ERR_CUDA;
+    return zl_coalesced_attn_bwd(t, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, ZL_NOALLOC_SCRATCH_BYTES, stream);
+}
+
 zl_status zl_set_kernel_timing(zl_tasks* t, int32_t enable) {
     if (!t) return ZL_ERR_INVALID_ARG;
     t->timing = enable != 0;
