@@ -189,7 +189,7 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 #define ZL_WAIT(bar, parity, site)                                        \
     do {                                                                  \
         ZL_PROF_T0                                                        \
-        if (!mbar_wait((bar), (parity), kWaitLimitNs) || sm.abort_flag) { \
+        if (!mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag)) { \
             report(p.status, &sm.abort_flag, 2000 + (site));              \
             goto teardown;                                                \
         }                                                                 \
@@ -198,7 +198,7 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 #define ZL_WAIT_WARP(bar, parity, site)                                              \
     do {                                                                             \
         ZL_PROF_T0                                                                   \
-        const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs) && !sm.abort_flag; \
+        const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag); \
         if (!__all_sync(0xffffffffu, ok_)) {                                         \
             report(p.status, &sm.abort_flag, 2000 + (site));                         \
             goto teardown;                                                           \

@@ -56,7 +56,7 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 // Wait used by a single elected thread.
 #define ZL_WAIT(bar, parity, site)                                        \
     do {                                                                  \
-        if (!mbar_wait((bar), (parity), kWaitLimitNs) || sm.abort_flag) { \
+        if (!mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag)) { \
             report(p.status, &sm.abort_flag, 1000 + (site));              \
             goto teardown;                                                \
         }                                                                 \
@@ -65,7 +65,7 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 // reconverges before the .sync.aligned TMEM instructions that follow.
 #define ZL_WAIT_WARP(bar, parity, site)                                              \
     do {                                                                             \
-        const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs) && !sm.abort_flag; \
+        const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag); \
         if (!__all_sync(0xffffffffu, ok_)) {                                         \
             report(p.status, &sm.abort_flag, 1000 + (site));                         \
             goto teardown;                                                           \

@@ -48,16 +48,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: polls until the phase with the given parity completes or `limit_ns` of
-// wall time has passed.  Returns false on expiry (the caller records the error and unwinds).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: polls until the phase with the given parity completes, `limit_ns` of wall time
+// has passed, or *abort_flag becomes non-zero (another role of the CTA gave up).  Returns false
+// in the last two cases; the caller records the error and unwinds.  The common case -- the phase
+// is already complete or completes within the first hardware-timed try -- costs one instruction.
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, uint64_t limit_ns,
+                                            const volatile int32_t* abort_flag) {
     const uint64_t t0 = globaltimer();
     uint32_t spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0x3FF) == 0 && globaltimer() - t0 > limit_ns) return false;
+        if ((++spins & 0xFF) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer() - t0 > limit_ns) return false;
+        }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns,
+                                          const volatile int32_t* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, limit_ns, abort_flag);
 }
 
 // ----------------------------------------------------------------------------- fences
