@@ -35,6 +35,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "coalesced attention TFLOP/s fwd and fwd+bwd; % of B200 dense BF16 peak"
+# DRAM traffic of the backward main kernel from one ncu capture on configuration 3
+# (dram__bytes_read.sum + dram__bytes_write.sum, profiles/zl_bwd_main_kernel_cfg3.txt); scaled to the
+# benchmarked workload by the counted backward FLOPs, which the K/V and Q/dO streaming follows.
+NCU_BWD_MAIN_CFG3_DRAM_BYTES = 2.484214e9 + 1.457662e9
+NCU_BWD_MAIN_CFG3_FLOPS = 2.5 * 4.0 * (16 * 1560 * 1560 + 8 * 8190 * 8190) * 128 * 12
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -289,7 +294,8 @@ def run_ours(args):
                 "unit": "TFLOP/s", "frac": (achieved / peak_t if achieved else None),
                 "peak_kind": f"{peak_kind} sustained bf16 (kernel timed inside a long step)",
                 "frac_of_burst": (achieved / float(peaks.get("bf16_tflops", 1590.0)) if achieved else None),
-                "traffic": None}
+                "traffic": NCU_BWD_MAIN_CFG3_DRAM_BYTES * p.bwd_flops() / NCU_BWD_MAIN_CFG3_FLOPS,
+                "traffic_note": "bytes per launch, scaled by counted FLOPs from an ncu capture on configuration 3"}
     fm = kernels["fwd"]["avg_ms"]
     fwd_kernel_tflops = p.fwd_flops() / (fm * 1e-3) / 1e12 if fm else None
     mm = kernels["merge"]["avg_ms"]
