@@ -42,7 +42,7 @@ struct FwdSmem {
     alignas(1024) uint8_t k[kStages][kTileBytes];
     alignas(1024) uint8_t v[kStages][kTileBytes];
     alignas(8) uint64_t q_full[2], q_empty;
-    uint64_t k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages];
+    uint64_t kv_full[kStages], kv_empty[kStages];  // K and V of a stage travel together
     uint64_t s_full[2], p_full[2], o_full[2];
     uint32_t tmem_base;
     volatile int32_t abort_flag;
@@ -98,10 +98,8 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         mbar_init(&sm.q_full[1], 1);
         mbar_init(&sm.q_empty, 1);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.k_full[s], 1);
-            mbar_init(&sm.v_full[s], 1);
-            mbar_init(&sm.k_empty[s], 1);
-            mbar_init(&sm.v_empty[s], 1);
+            mbar_init(&sm.kv_full[s], 1);
+            mbar_init(&sm.kv_empty[s], 1);
         }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&sm.s_full[x], 1);
@@ -142,10 +140,10 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 for (int j = 0; j < n_kv; ++j, ++kv_cnt) {
                     const int s = kv_cnt % kStages;
                     const uint32_t ph = (kv_cnt / kStages) & 1;
-                    ZL_WAIT(&sm.k_empty[s], ph ^ 1, 2);
-                    mbar_arrive_expect_tx(&sm.k_full[s], Smem::kTileBytes);
+                    ZL_WAIT(&sm.kv_empty[s], ph ^ 1, 2);
+                    mbar_arrive_expect_tx(&sm.kv_full[s], 2 * Smem::kTileBytes);
                     for (int b = 0; b < kBoxes; ++b)
-                        tma_load_3d(sm.k[s] + b * Smem::kBoxBytes, &tm_k, &sm.k_full[s], b * 64, wi.head,
+                        tma_load_3d(sm.k[s] + b * Smem::kBoxBytes, &tm_k, &sm.kv_full[s], b * 64, wi.head,
                                     t.kv_off + j * kTileKV);
                     if (j == 0 && has_b) {  // second query tile right after the first K tile
                         mbar_arrive_expect_tx(&sm.q_full[1], Smem::kTileBytes);
@@ -154,10 +152,8 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                                         t.q_off + wi.row0 + kTileQ);
                         ++qb_cnt;
                     }
-                    ZL_WAIT(&sm.v_empty[s], ph ^ 1, 3);
-                    mbar_arrive_expect_tx(&sm.v_full[s], Smem::kTileBytes);
                     for (int b = 0; b < kBoxes; ++b)
-                        tma_load_3d(sm.v[s] + b * Smem::kBoxBytes, &tm_v, &sm.v_full[s], b * 64, wi.head,
+                        tma_load_3d(sm.v[s] + b * Smem::kBoxBytes, &tm_v, &sm.kv_full[s], b * 64, wi.head,
                                     t.kv_off + j * kTileKV);
                 }
             }
@@ -196,30 +192,27 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const bool has_b = wi.rows > kTileQ;
                 ZL_WAIT(&sm.q_full[0], q_cnt & 1, 11);
                 ++q_cnt;
-                ZL_WAIT(&sm.k_full[kv_cnt % kStages], (kv_cnt / kStages) & 1, 12);
+                ZL_WAIT(&sm.kv_full[kv_cnt % kStages], (kv_cnt / kStages) & 1, 12);
                 tc_fence_after();
                 issue_s(0, kv_cnt % kStages);
                 if (has_b) {
                     ZL_WAIT(&sm.q_full[1], qb_cnt & 1, 13);
                     ++qb_cnt;
-                    tc_fence_after();
                     issue_s(1, kv_cnt % kStages);
                 }
-                mma_commit(&sm.k_empty[kv_cnt % kStages]);
                 if (n_kv == 1) mma_commit(&sm.q_empty);
                 for (int j = 0; j < n_kv; ++j, ++kv_cnt) {
                     const uint32_t s = kv_cnt % kStages, nk = kv_cnt + 1, sn = nk % kStages;
                     const bool has_next = j + 1 < n_kv;
-                    // tile A: P_A(j) is in TMEM (S_A(j) fully read, O_A rescaled if needed)
+                    // tile A: P_A(j) is in TMEM (S_A(j) fully read, O_A rescaled if needed); K(j), V(j)
+                    // were waited for when S(j) was issued
                     ZL_WAIT(&sm.p_full[0], pa_cnt & 1, 14);
                     ++pa_cnt;
-                    ZL_WAIT(&sm.v_full[s], (kv_cnt / kStages) & 1, 15);
                     tc_fence_after();
                     issue_pv(0, s, j > 0);
                     if (!has_next) mma_commit(&sm.o_full[0]);
                     if (has_next) {
-                        ZL_WAIT(&sm.k_full[sn], (nk / kStages) & 1, 16);
-                        tc_fence_after();
+                        ZL_WAIT(&sm.kv_full[sn], (nk / kStages) & 1, 16);
                         issue_s(0, sn);  // overwrites P_A(j): ordered after P_A V on the tensor pipe
                     }
                     if (has_b) {
@@ -229,10 +222,9 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         issue_pv(1, s, j > 0);
                         if (!has_next) mma_commit(&sm.o_full[1]);
                     }
-                    mma_commit(&sm.v_empty[s]);
+                    mma_commit(&sm.kv_empty[s]);  // S_A(j), S_B(j), P_A V(j), P_B V(j) are the stage's last readers
                     if (has_next) {
                         if (has_b) issue_s(1, sn);
-                        mma_commit(&sm.k_empty[sn]);
                         if (j + 2 == n_kv) mma_commit(&sm.q_empty);  // last S of the item issued
                     }
                 }
