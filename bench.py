@@ -459,6 +459,52 @@ def run_reference(args):
     print(json.dumps(out), flush=True)
 
 
+def run_ablation(args):
+    """Extra measurements that evidence design choices (printed as one JSON line, not the headline):
+    'straggler' -- config 3's images next to one WHOLE 32,760-token video (the naive data-parallel
+    placement): forward time with the work list longest-first, in placement order and shortest-first;
+    'coalescing' -- config 2 as one coalesced launch vs one launch per sequence."""
+    import torch
+    import zl_workloads as W
+    import paper_2608_01150_b200 as Z
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    out = {"ablation": args.ablation}
+    if args.ablation == "straggler":
+        p = W.straggler_placement()
+        wl = Workload(p, device)
+        for name, mode in (("longest_first", 0), ("placement_order", 1), ("shortest_first", 2)):
+            wl.h.set_fwd_order(mode)
+            for _ in range(3):
+                wl.fwd()
+            ms = wl.time_region(wl.fwd, 10) / 10
+            out[name] = {"fwd_ms": ms, "fwd_tflops": p.fwd_flops() / ms / 1e9}
+        wl.h.set_fwd_order(0)
+    else:
+        p = W.config(2)
+        wl = Workload(p, device)
+        for _ in range(3):
+            wl.fwd()
+        ms = wl.time_region(wl.fwd, 10) / 10
+        out["coalesced"] = {"launches": 1, "fwd_ms": ms, "fwd_tflops": p.fwd_flops() / ms / 1e9}
+        # the same sequences, one launch each (handles built beforehand)
+        H, d = p.n_heads, p.head_dim
+        hs = []
+        for i in range(p.n_whole):
+            a, b = p.cu_seqlens[i], p.cu_seqlens[i + 1]
+            hs.append((a, b, Z.build_tasks([0, b - a], [], b - a, b - a, H, d)))
+
+        def per_sequence():
+            for a, b, h in hs:
+                Z.coalesced_attn_fwd(h, wl.Q[a:b], wl.K[a:b], wl.V[a:b], p.scale, wl.O[a:b], wl.LSE, None, None)
+        # LSE is [H, total_q]: a per-sequence handle writes rows [0, len) of each head's line; only timing matters here
+        for _ in range(3):
+            per_sequence()
+        ms = wl.time_region(per_sequence, 10) / 10
+        out["per_sequence"] = {"launches": len(hs), "fwd_ms": ms, "fwd_tflops": p.fwd_flops() / ms / 1e9}
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -468,7 +514,13 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="named configuration 1..5 (default: Wan-14B-shaped rank)")
     ap.add_argument("--extra-configs", default="2,3,5", help="also time these configurations (N=1 only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ablation", default="", choices=["", "straggler", "coalescing"],
+                    help="print an extra measurement instead of the benchmark line")
     args = ap.parse_args()
+
+    if args.ablation:
+        run_ablation(args)
+        return
 
     if args.impl == "reference":
         run_reference(args)

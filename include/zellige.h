@@ -205,6 +205,20 @@ zl_status zl_set_kernel_timing(zl_tasks* tasks, int32_t enable);
 zl_status zl_get_kernel_timing(zl_tasks* tasks, float* total_ms /* [ZL_K_COUNT] */,
                                int32_t* launches /* [ZL_K_COUNT] */);
 
+/* Measurement / diagnosis aids (no paper counterpart).
+ *
+ * zl_debug_set_fwd_order re-sorts the handle's forward work list and uploads it: 0 = longest-first
+ * (the default built by zl_build_tasks), 1 = placement order (task, head, block), 2 = shortest-first.
+ * Results never depend on the order; it exists to measure what longest-first ordering buys.
+ *
+ * zl_selftest_bounded_wait launches a one-CTA kernel that waits, with the same bounded wait the
+ * attention kernels use, on an mbarrier nobody ever arrives on, with a limit of `limit_us`
+ * microseconds (clamped to [1, 100000]).  The wait must expire: the kernel then records
+ * ZL_ERR_TIMEOUT in the handle's device status word and returns normally, which
+ * zl_last_device_status reports.  Nothing hangs and nothing faults. */
+zl_status zl_debug_set_fwd_order(zl_tasks* tasks, int32_t mode, void* stream);
+zl_status zl_selftest_bounded_wait(const zl_tasks* tasks, int32_t limit_us, void* stream);
+
 const char* zl_status_str(zl_status s);
 
 /* Number of this library's kernel launches enqueued since load (all handles). */

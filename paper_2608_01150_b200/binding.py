@@ -77,6 +77,10 @@ def _load():
     lib.zl_set_kernel_timing.argtypes = [vp, i32]
     lib.zl_get_kernel_timing.restype = ctypes.c_int
     lib.zl_get_kernel_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+    lib.zl_debug_set_fwd_order.restype = ctypes.c_int
+    lib.zl_debug_set_fwd_order.argtypes = [vp, i32, vp]
+    lib.zl_selftest_bounded_wait.restype = ctypes.c_int
+    lib.zl_selftest_bounded_wait.argtypes = [vp, i32, vp]
     lib.zl_status_str.restype = ctypes.c_char_p
     lib.zl_status_str.argtypes = [ctypes.c_int]
     lib.zl_launch_count.restype = ctypes.c_int64
@@ -161,6 +165,14 @@ class TaskHandle:
         n = (ctypes.c_int32 * len(KERNEL_NAMES))()
         _check(_lib.zl_get_kernel_timing(self._ptr, ms, n), "zl_get_kernel_timing")
         return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(KERNEL_NAMES)}
+
+    def set_fwd_order(self, mode: int, stream=None):
+        """0 longest-first (default), 1 placement order, 2 shortest-first (measurement aid)."""
+        _check(_lib.zl_debug_set_fwd_order(self._ptr, mode, _stream_ptr(stream)), "zl_debug_set_fwd_order")
+
+    def selftest_bounded_wait(self, limit_us: int = 1000, stream=None):
+        """Launches a kernel whose bounded wait must expire; read the outcome with last_device_status()."""
+        _check(_lib.zl_selftest_bounded_wait(self._ptr, limit_us, _stream_ptr(stream)), "zl_selftest_bounded_wait")
 
     def close(self):
         if self._ptr:

@@ -2,12 +2,14 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <tuple>
 
 #include "zl_device.h"
 
@@ -471,6 +473,40 @@ zl_status zl_coalesced_attn_bwd_noalloc(const zl_tasks* t, const void* q, const 
     void* scratch = noalloc_scratch_for(dev);
     if (!scratch) return ZL_ERR_CUDA;
     return zl_coalesced_attn_bwd(t, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, ZL_NOALLOC_SCRATCH_BYTES, stream);
+}
+
+zl_status zl_debug_set_fwd_order(zl_tasks* t, int32_t mode, void* stream) {
+    if (!t || mode < 0 || mode > 2) return ZL_ERR_INVALID_ARG;
+    Schedule& s = t->sched;
+    auto placement_order = [](const WorkItem& a, const WorkItem& b) {
+        return std::tie(a.unit, a.head, a.row0) < std::tie(b.unit, b.head, b.row0);
+    };
+    std::stable_sort(s.fwd_items.begin(), s.fwd_items.end(), placement_order);
+    if (mode != 1) {
+        std::stable_sort(s.fwd_items.begin(), s.fwd_items.end(), [&](const WorkItem& a, const WorkItem& b) {
+            const int32_t ka = s.tasks[a.unit].kv_len, kb = s.tasks[b.unit].kv_len;
+            if (ka != kb) return mode == 0 ? ka > kb : ka < kb;
+            if (a.rows != b.rows) return mode == 0 ? a.rows > b.rows : a.rows < b.rows;
+            return false;
+        });
+    }
+    if (t->device < 0 || s.fwd_items.empty()) return ZL_OK;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(t->d_fwd_items, s.fwd_items.data(), s.fwd_items.size() * sizeof(WorkItem),
+                        cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaStreamSynchronize(cs) != cudaSuccess)
+        return ZL_ERR_CUDA;
+    return ZL_OK;
+}
+
+zl_status zl_selftest_bounded_wait(const zl_tasks* t, int32_t limit_us, void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    if (t->device < 0) return ZL_ERR_CUDA;
+    const int32_t us = limit_us < 1 ? 1 : (limit_us > 100000 ? 100000 : limit_us);
+    if (launch_wait_selftest(t->d_status, (uint64_t)us * 1000ull, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return ZL_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return ZL_OK;
 }
 
 zl_status zl_set_kernel_timing(zl_tasks* t, int32_t enable) {

@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 
 #include "zl_device.h"
+#include "zl_ptx.cuh"
 
 namespace zl {
 
@@ -87,6 +88,31 @@ cudaError_t launch_merge(int head_dim, const MergeParams& p, int n_sms, cudaStre
         zl_merge_kernel<128><<<grid, kMergeThreads, 0, stream>>>(p);
     else
         zl_merge_kernel<64><<<grid, kMergeThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+// Self-test of the bounded wait: a barrier that never completes must time out, be reported through
+// the status word, and leave the context usable.
+namespace {
+__global__ void zl_wait_selftest_kernel(int32_t* status, uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ volatile int32_t abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (!ptx::mbar_wait(&bar, 0, limit_ns, &abort_flag)) {
+            if (atomicCAS(status, 0, (int)ZL_ERR_TIMEOUT) == 0) status[1] = 9001;
+        }
+    }
+}
+}  // namespace
+
+cudaError_t launch_wait_selftest(int32_t* status, uint64_t limit_ns, cudaStream_t stream) {
+    zl_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
     return cudaGetLastError();
 }
 

@@ -135,3 +135,31 @@ def test_randomised_small_placements():
         Kb = random_bits(rng, p.total_kv, H, d)
         Vb = random_bits(rng, p.total_kv, H, d)
         _run(p, Qb, Kb, Vb)
+
+
+def test_bounded_wait_expires_and_is_reported():
+    """A wait nobody satisfies returns after its limit, reports ZL_ERR_TIMEOUT through the device status
+    word and leaves the context usable (no trap, no hang)."""
+    p = W.config(1)
+    run = GpuRun(p)
+    run.h.selftest_bounded_wait(limit_us=500)
+    torch.cuda.synchronize()
+    code, where = run.h.last_device_status()
+    assert (code, where) == (6, 9001)            # ZL_ERR_TIMEOUT at the self-test site
+    assert run.h.last_device_status() == (0, 0)  # reading clears the word
+    Qd, Kd, Vd = to_dev(bits(p, "Q")), to_dev(bits(p, "K")), to_dev(bits(p, "V"))
+    O, LSE, _, _ = run.forward(Qd, Kd, Vd)       # the same handle and context still work
+    assert torch.isfinite(O.float()).all()
+
+
+def test_results_do_not_depend_on_the_work_order():
+    p = W.make_placement("order", 2, 128, 5, [700, 130, 1000], [(1, 2, 300)])
+    rng = np.random.RandomState(8)
+    Qd = to_dev(random_bits(rng, p.total_q, 2, 128)); Kd = to_dev(random_bits(rng, p.total_kv, 2, 128))
+    Vd = to_dev(random_bits(rng, p.total_kv, 2, 128))
+    run = GpuRun(p)
+    ref = run.forward(Qd, Kd, Vd)
+    for mode in (1, 2, 0):
+        run.h.set_fwd_order(mode)
+        out = run.forward(Qd, Kd, Vd)
+        assert torch.equal(out[0], ref[0]) and torch.equal(out[1], ref[1])
