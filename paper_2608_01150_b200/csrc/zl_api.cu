@@ -103,7 +103,7 @@ bool make_tmap_f32_acc(CUtensorMap* m, const void* base, int64_t rows, int n_hea
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)(rows > 0 ? rows : 1)};
     cuuint64_t strides[2] = {(cuuint64_t)head_dim * 4, (cuuint64_t)head_dim * 4 * n_heads};
-    cuuint32_t box[3] = {32, 1, 128};
+    cuuint32_t box[3] = {32, 1, 32};  // one warp's 32 query rows x 32 fp32 columns
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,

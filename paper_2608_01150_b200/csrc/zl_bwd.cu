@@ -313,8 +313,12 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     }
                 }
             }
-        } else if (warp == 1 && lane == 0) {
+        } else if (warp == 1) {
             // -------------------------------------------------------------- MMA issuer
+            // The whole warp runs this loop converged and one elected lane issues: descriptors
+            // and barrier addresses then stay warp-uniform, which makes commits and satisfied
+            // waits several times cheaper than from a single diverged thread.
+            const bool mma_lane = elect_one();
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: K-major x K-major
             constexpr uint32_t idesc_dv = make_idesc_bf16(128, D, 0, 1);    // A in TMEM / K-major smem, B MN-major
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 1, 1);    // A MN-major smem, B MN-major
@@ -340,10 +344,10 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
-                    mma_ss(tmem + kColS, dk_k + off, dq + off, idesc_s, ks > 0);
+                    if (mma_lane) mma_ss(tmem + kColS, dk_k + off, dq + off, idesc_s, ks > 0);
                 }
-                mma_ss(tmem + kColS, dones_s, daug0 + stage * kAugStageStep, idesc_s, true);
-                mma_commit(&sm.s_full);
+                if (mma_lane) mma_ss(tmem + kColS, dones_s, daug0 + stage * kAugStageStep, idesc_s, true);
+                if (mma_lane) mma_commit(&sm.s_full);
                 ZL_PROF_SEG_END(40)
             };
             // dP^T = V dO^T - D: the ones sit in the second K chunk, where the tile holds the D pieces
@@ -352,19 +356,19 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
-                    mma_ss(tmem + kColDP, dv_k + off, ddo_k + off, idesc_s, ks > 0);
+                    if (mma_lane) mma_ss(tmem + kColDP, dv_k + off, ddo_k + off, idesc_s, ks > 0);
                 }
-                mma_ss(tmem + kColDP, dones_dp, daug0 + stage * kAugStageStep, idesc_s, true);
-                mma_commit(&sm.dp_full);
+                if (mma_lane) mma_ss(tmem + kColDP, dones_dp, daug0 + stage * kAugStageStep, idesc_s, true);
+                if (mma_lane) mma_commit(&sm.dp_full);
                 ZL_PROF_SEG_END(41)
             };
             auto issue_dv = [&](bool acc) {
                 ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
-                    mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8, ddo_mn + ks * (2048 >> 4), idesc_dv,
+                    if (mma_lane) mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8, ddo_mn + ks * (2048 >> 4), idesc_dv,
                            acc || ks > 0);
-                mma_commit(&sm.do_empty);
+                if (mma_lane) mma_commit(&sm.do_empty);
                 ZL_PROF_SEG_END(42)
             };
             uint32_t item_cnt = 0, it_cnt = 0;
@@ -372,29 +376,29 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
                 const int n_it = count_q_tiles(p, g);
-                ZL_WAIT(&sm.kv_full, item_cnt & 1, 11);
+                ZL_WAIT_WARP(&sm.kv_full, item_cnt & 1, 11);
                 // prologue: S, dP, dV of the item's first query tile and S of the second.
                 // Steady-state order on the tensor pipe: dK(i) dQ(i) dP(i+1) dV(i+1) S(i+2).
-                ZL_WAIT(&sm.q_full[it_cnt & 1], (it_cnt >> 1) & 1, 12);
+                ZL_WAIT_WARP(&sm.q_full[it_cnt & 1], (it_cnt >> 1) & 1, 12);
                 tc_fence_after();
                 issue_s(it_cnt & 1);
-                ZL_WAIT(&sm.do_full, it_cnt & 1, 13);
-                ZL_WAIT(&sm.dq_empty, (it_cnt & 1) ^ 1, 14);  // previous dQ tile drained from the dP columns
+                ZL_WAIT_WARP(&sm.do_full, it_cnt & 1, 13);
+                ZL_WAIT_WARP(&sm.dq_empty, (it_cnt & 1) ^ 1, 14);  // previous dQ tile drained from the dP columns
                 tc_fence_after();
                 issue_dp(it_cnt & 1);
-                ZL_WAIT(&sm.p_full, it_cnt & 1, 15);
+                ZL_WAIT_WARP(&sm.p_full, it_cnt & 1, 15);
                 tc_fence_after();
                 issue_dv(false);
                 if (n_it > 1) {
                     const uint32_t n1 = it_cnt + 1;
-                    ZL_WAIT(&sm.q_full[n1 & 1], (n1 >> 1) & 1, 16);
+                    ZL_WAIT_WARP(&sm.q_full[n1 & 1], (n1 >> 1) & 1, 16);
                     tc_fence_after();
                     issue_s(n1 & 1);  // overwrites P^T: ordered after dV on the tensor pipe
                 }
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     const uint64_t dq_mn = dq_mn0 + (it_cnt & 1) * kQStageStep;
                     ZL_TRACE(0, 0, it_cnt)
-                    ZL_WAIT(&sm.ds_full, it_cnt & 1, 17);
+                    ZL_WAIT_WARP(&sm.ds_full, it_cnt & 1, 17);
                     ZL_TRACE(0, 1, it_cnt)
                     tc_fence_after();
                     {
@@ -402,34 +406,34 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
                             const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
-                            mma_ss(tmem + kColDK, dds_k + off, dq_mn + ks * (2048 >> 4), idesc_dv, i > 0 || ks > 0);
+                            if (mma_lane) mma_ss(tmem + kColDK, dds_k + off, dq_mn + ks * (2048 >> 4), idesc_dv, i > 0 || ks > 0);
                         }
-                        mma_commit(&sm.q_empty[it_cnt & 1]);  // Q stage free early: its reload has dQ, dP, dV to land
+                        if (mma_lane) mma_commit(&sm.q_empty[it_cnt & 1]);  // Q stage free early: its reload has dQ, dP, dV to land
                         ZL_TRACE(0, 2, it_cnt)
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
-                            mma_ss(tmem + kColDP, dds_mn + ks * (2048 >> 4), dk_mn + ks * (2048 >> 4), idesc_dq, ks > 0);
-                        mma_commit(&sm.dq_full);
-                        mma_commit(&sm.ds_free);
+                            if (mma_lane) mma_ss(tmem + kColDP, dds_mn + ks * (2048 >> 4), dk_mn + ks * (2048 >> 4), idesc_dq, ks > 0);
+                        if (mma_lane) mma_commit(&sm.dq_full);
+                        if (mma_lane) mma_commit(&sm.ds_free);
                         ZL_PROF_SEG_END(43)
                     }
                     ZL_TRACE(0, 3, it_cnt)
                     if (i + 1 < n_it) {
                         const uint32_t n1 = it_cnt + 1, n2 = it_cnt + 2;
-                        ZL_WAIT(&sm.do_full, n1 & 1, 18);
+                        ZL_WAIT_WARP(&sm.do_full, n1 & 1, 18);
                         ZL_TRACE(0, 4, it_cnt)
-                        ZL_WAIT(&sm.dq_empty, it_cnt & 1, 19);
+                        ZL_WAIT_WARP(&sm.dq_empty, it_cnt & 1, 19);
                         ZL_TRACE(0, 5, it_cnt)
                         tc_fence_after();
                         issue_dp(n1 & 1);
                         ZL_TRACE(0, 6, it_cnt)
-                        ZL_WAIT(&sm.p_full, n1 & 1, 20);
+                        ZL_WAIT_WARP(&sm.p_full, n1 & 1, 20);
                         ZL_TRACE(0, 7, it_cnt)
                         tc_fence_after();
                         issue_dv(true);
                         ZL_TRACE(0, 8, it_cnt)
                         if (i + 2 < n_it) {
-                            ZL_WAIT(&sm.q_full[n2 & 1], (n2 >> 1) & 1, 16);
+                            ZL_WAIT_WARP(&sm.q_full[n2 & 1], (n2 >> 1) & 1, 16);
                             ZL_TRACE(0, 9, it_cnt)
                             tc_fence_after();
                             issue_s(n2 & 1);
@@ -437,8 +441,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         }
                     }
                 }
-                mma_commit(&sm.acc_full);
-                mma_commit(&sm.kv_empty);
+                if (mma_lane) mma_commit(&sm.acc_full);
+                if (mma_lane) mma_commit(&sm.kv_empty);
             }
         }
     } else if (warp < 12) {
@@ -585,7 +589,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-        const bool leader = (warp == 12 && lane == 0);
+        const bool leader = (lane == 0);  // per warp
         uint32_t it_cnt = 0, chunk_cnt = 0;
         for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
             const WorkItem wi = p.items[it];
@@ -615,20 +619,22 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (warp == 12 && lane == 0) { ZL_TRACE(2, 2, it_cnt) }
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c, ++chunk_cnt) {
-                            uint8_t* buf = sm.dq_stage;
+                            // each warp stages its own 32 rows and adds them with its own reduce: no
+                            // warpgroup barrier, and the four streams overlap in the copy engine
+                            uint8_t* buf = sm.dq_stage + quarter * 4096;
                             if (chunk_cnt >= 1) {
                                 if (leader) bulk_wait_group_read<0>();  // the previous reduce has read the buffer
-                                named_bar_sync(1, 128);
+                                __syncwarp();
                             }
-                            const uint32_t row_addr = smem_u32(buf) + row * 128;
+                            const uint32_t row_addr = smem_u32(buf) + lane * 128;
 #pragma unroll
                             for (int k4 = 0; k4 < 8; ++k4)
-                                st_shared_v4(row_addr + ((k4 ^ (row & 7)) << 4), r[c * 32 + k4 * 4], r[c * 32 + k4 * 4 + 1],
+                                st_shared_v4(row_addr + ((k4 ^ (lane & 7)) << 4), r[c * 32 + k4 * 4], r[c * 32 + k4 * 4 + 1],
                                              r[c * 32 + k4 * 4 + 2], r[c * 32 + k4 * 4 + 3]);
                             fence_proxy_async_smem();
-                            named_bar_sync(1, 128);
+                            __syncwarp();
                             if (leader) {
-                                tma_reduce_add_3d(&tm_dq, buf, c * 32, wi.head, t.q_slot + qt * kTileQ);
+                                tma_reduce_add_3d(&tm_dq, buf, c * 32, wi.head, t.q_slot + qt * kTileQ + quarter * 32);
                                 bulk_commit_group();
                             }
                         }
