@@ -165,18 +165,29 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 #ifdef ZL_PROFILE
 // Development aid (profile builds only): cycles spent waiting at each site and in each MMA
 // issue segment, for the first CTAs.
+#ifdef ZL_TRACE_ONLY
+#define ZL_PROF_T0
+#define ZL_PROF_ADD(site)
+#define ZL_PROF_MARK(site)
+#else
 #define ZL_PROF_T0 const long long prof_t0_ = clock64();
 #define ZL_PROF_ADD(site) \
     if (p.prof && blockIdx.x < 4 && lane == 0) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_t0_));
 #define ZL_PROF_MARK(site) \
     if (p.prof && blockIdx.x < 4 && warp == 4 && lane == 0) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_seg_));
+#endif
 // Event trace: timestamp of event `ev` (0..15) of role `role` (0 MMA, 1 P/dS warp 4, 2 dQ warp 12) for
 // global iterations 200..207 of CTA 0.
 #define ZL_TRACE(role, ev, itc) \
     if (p.prof && blockIdx.x == 0 && (itc) >= 200u && (itc) < 208u) p.prof[256 + (role) * 128 + ((itc) - 200u) * 16 + (ev)] = clock64();
+#ifdef ZL_TRACE_ONLY
+#define ZL_PROF_SEG_BEGIN
+#define ZL_PROF_SEG_END(site)
+#else
 #define ZL_PROF_SEG_BEGIN const long long prof_seg_ = clock64();
 #define ZL_PROF_SEG_END(site) \
     if (p.prof && blockIdx.x < 4) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_seg_));
+#endif
 #else
 #define ZL_PROF_T0
 #define ZL_PROF_ADD(site)
