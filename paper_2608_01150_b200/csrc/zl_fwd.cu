@@ -157,8 +157,11 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                                     t.kv_off + j * kTileKV);
                 }
             }
-        } else if (warp == 1 && lane == 0) {
+        } else if (warp == 1) {
             // -------------------------------------------------------------- MMA issuer
+            // The whole warp runs this loop converged and one elected lane issues, which keeps
+            // descriptors and barrier addresses warp-uniform (cheaper commits and satisfied waits).
+            const bool mma_lane = elect_one();
             constexpr uint32_t idesc_s = make_idesc_bf16(kTileQ, kTileKV, 0, 0);
             constexpr uint32_t idesc_o = make_idesc_bf16(kTileQ, D, 0, 1);
             const uint64_t dq0 = make_desc_sw128(smem_u32(sm.q[0]), 16, 1024);
@@ -171,16 +174,16 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
-                    mma_ss(tmem + kColS + x * 128, dq + off, dk + off, idesc_s, ks > 0);
+                    if (mma_lane) mma_ss(tmem + kColS + x * 128, dq + off, dk + off, idesc_s, ks > 0);
                 }
-                mma_commit(&sm.s_full[x]);
+                if (mma_lane) mma_commit(&sm.s_full[x]);
             };
             // O_x (+)= P_x V
             auto issue_pv = [&](int x, uint32_t stage, bool acc) {
                 const uint64_t dv = dv0 + stage * kTileStep;
 #pragma unroll
                 for (int ks = 0; ks < kTileKV / 16; ++ks)
-                    mma_ts(tmem + kColO + x * 128, tmem + kColS + x * 128 + ks * 8, dv + ks * (2048 >> 4), idesc_o,
+                    if (mma_lane) mma_ts(tmem + kColO + x * 128, tmem + kColS + x * 128 + ks * 8, dv + ks * (2048 >> 4), idesc_o,
                            acc || ks > 0);
             };
             uint32_t q_cnt = 0, qb_cnt = 0, kv_cnt = 0, pa_cnt = 0, pb_cnt = 0;
@@ -190,42 +193,42 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const int n_kv = (t.kv_len + kTileKV - 1) / kTileKV;
                 if (n_kv == 0) continue;
                 const bool has_b = wi.rows > kTileQ;
-                ZL_WAIT(&sm.q_full[0], q_cnt & 1, 11);
+                ZL_WAIT_WARP(&sm.q_full[0], q_cnt & 1, 11);
                 ++q_cnt;
-                ZL_WAIT(&sm.kv_full[kv_cnt % kStages], (kv_cnt / kStages) & 1, 12);
+                ZL_WAIT_WARP(&sm.kv_full[kv_cnt % kStages], (kv_cnt / kStages) & 1, 12);
                 tc_fence_after();
                 issue_s(0, kv_cnt % kStages);
                 if (has_b) {
-                    ZL_WAIT(&sm.q_full[1], qb_cnt & 1, 13);
+                    ZL_WAIT_WARP(&sm.q_full[1], qb_cnt & 1, 13);
                     ++qb_cnt;
                     issue_s(1, kv_cnt % kStages);
                 }
-                if (n_kv == 1) mma_commit(&sm.q_empty);
+                if (n_kv == 1) if (mma_lane) mma_commit(&sm.q_empty);
                 for (int j = 0; j < n_kv; ++j, ++kv_cnt) {
                     const uint32_t s = kv_cnt % kStages, nk = kv_cnt + 1, sn = nk % kStages;
                     const bool has_next = j + 1 < n_kv;
                     // tile A: P_A(j) is in TMEM (S_A(j) fully read, O_A rescaled if needed); K(j), V(j)
                     // were waited for when S(j) was issued
-                    ZL_WAIT(&sm.p_full[0], pa_cnt & 1, 14);
+                    ZL_WAIT_WARP(&sm.p_full[0], pa_cnt & 1, 14);
                     ++pa_cnt;
                     tc_fence_after();
                     issue_pv(0, s, j > 0);
-                    if (!has_next) mma_commit(&sm.o_full[0]);
+                    if (!has_next) if (mma_lane) mma_commit(&sm.o_full[0]);
                     if (has_next) {
-                        ZL_WAIT(&sm.kv_full[sn], (nk / kStages) & 1, 16);
+                        ZL_WAIT_WARP(&sm.kv_full[sn], (nk / kStages) & 1, 16);
                         issue_s(0, sn);  // overwrites P_A(j): ordered after P_A V on the tensor pipe
                     }
                     if (has_b) {
-                        ZL_WAIT(&sm.p_full[1], pb_cnt & 1, 17);
+                        ZL_WAIT_WARP(&sm.p_full[1], pb_cnt & 1, 17);
                         ++pb_cnt;
                         tc_fence_after();
                         issue_pv(1, s, j > 0);
-                        if (!has_next) mma_commit(&sm.o_full[1]);
+                        if (!has_next) if (mma_lane) mma_commit(&sm.o_full[1]);
                     }
-                    mma_commit(&sm.kv_empty[s]);  // S_A(j), S_B(j), P_A V(j), P_B V(j) are the stage's last readers
+                    if (mma_lane) mma_commit(&sm.kv_empty[s]);  // S_A(j), S_B(j), P_A V(j), P_B V(j) are the stage's last readers
                     if (has_next) {
                         if (has_b) issue_s(1, sn);
-                        if (j + 2 == n_kv) mma_commit(&sm.q_empty);  // last S of the item issued
+                        if (j + 2 == n_kv) if (mma_lane) mma_commit(&sm.q_empty);  // last S of the item issued
                     }
                 }
             }
