@@ -296,6 +296,14 @@ zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k,
     p.o_partial = o_partial;
     p.lse_partial = lse_partial;
     p.status = t->d_status;
+#ifdef ZL_PROFILE
+    static long long* d_fprof = nullptr;
+    if (getenv("ZL_PROF")) {
+        if (!d_fprof) cudaMalloc(&d_fprof, 1024 * sizeof(long long));
+        cudaMemsetAsync(d_fprof, 0, 1024 * sizeof(long long), static_cast<cudaStream_t>(stream));
+        p.prof = d_fprof;
+    }
+#endif
     const int grid = std::min<int>(t->n_sms, p.n_items);
     {
         LaunchTimer lt(t, ZL_K_FWD, static_cast<cudaStream_t>(stream));
@@ -303,6 +311,23 @@ zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k,
             return ZL_ERR_CUDA;
     }
     g_launches.fetch_add(1);
+#ifdef ZL_PROFILE
+    if (p.prof && getenv("ZL_TRACE")) {
+        long long hprof[1024];
+        cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+        cudaMemcpy(hprof, p.prof, sizeof(hprof), cudaMemcpyDeviceToHost);
+        const long long t0 = hprof[256 + 0];
+        for (int role = 0; role < 3; ++role)
+            for (int itx = 0; itx < 8; ++itx) {
+                fprintf(stderr, "[zl fwd trace] role %d it %d:", role, 200 + itx);
+                for (int ev = 0; ev < 11; ++ev) {
+                    const long long v = hprof[256 + role * 128 + itx * 16 + ev];
+                    if (v) fprintf(stderr, " e%d=%lld", ev, v - t0);
+                }
+                fprintf(stderr, "\n");
+            }
+    }
+#endif
     return ZL_OK;
 }
 

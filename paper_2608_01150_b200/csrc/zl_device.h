@@ -22,6 +22,7 @@ struct FwdParams {
     float* o_partial;
     float* lse_partial;
     int32_t* status;  // [0] = code, [1] = where
+    long long* prof;  // development aid (ZL_PROFILE builds), else null
 };
 
 struct MergeParams {

@@ -53,6 +53,15 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
     if (atomicCAS(status, 0, (int)ZL_ERR_TIMEOUT) == 0) status[1] = where;
 }
 
+#ifdef ZL_PROFILE
+// Development aid (profile builds only): timestamps of event `ev` of role `role` (0 MMA warp,
+// 1 / 2 softmax warp 4 / 8) for key-tile iterations 200..207 of CTA 0.
+#define ZL_TRACE(role, ev, itc) \
+    if (p.prof && blockIdx.x == 0 && lane == 0 && (itc) >= 200u && (itc) < 208u) p.prof[256 + (role) * 128 + ((itc) - 200u) * 16 + (ev)] = clock64();
+#else
+#define ZL_TRACE(role, ev, itc)
+#endif
+
 // Wait used by a single elected thread.
 #define ZL_WAIT(bar, parity, site)                                        \
     do {                                                                  \
@@ -209,25 +218,33 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     const bool has_next = j + 1 < n_kv;
                     // tile A: P_A(j) is in TMEM (S_A(j) fully read, O_A rescaled if needed); K(j), V(j)
                     // were waited for when S(j) was issued
+                    ZL_TRACE(0, 0, kv_cnt)
                     ZL_WAIT_WARP(&sm.p_full[0], pa_cnt & 1, 14);
+                    ZL_TRACE(0, 1, kv_cnt)
                     ++pa_cnt;
                     tc_fence_after();
                     issue_pv(0, s, j > 0);
+                    ZL_TRACE(0, 2, kv_cnt)
                     if (!has_next) if (mma_lane) mma_commit(&sm.o_full[0]);
                     if (has_next) {
                         ZL_WAIT_WARP(&sm.kv_full[sn], (nk / kStages) & 1, 16);
+                        ZL_TRACE(0, 3, kv_cnt)
                         issue_s(0, sn);  // overwrites P_A(j): ordered after P_A V on the tensor pipe
+                        ZL_TRACE(0, 4, kv_cnt)
                     }
                     if (has_b) {
                         ZL_WAIT_WARP(&sm.p_full[1], pb_cnt & 1, 17);
+                        ZL_TRACE(0, 5, kv_cnt)
                         ++pb_cnt;
                         tc_fence_after();
                         issue_pv(1, s, j > 0);
+                        ZL_TRACE(0, 6, kv_cnt)
                         if (!has_next) if (mma_lane) mma_commit(&sm.o_full[1]);
                     }
                     if (mma_lane) mma_commit(&sm.kv_empty[s]);  // S_A(j), S_B(j), P_A V(j), P_B V(j) are the stage's last readers
                     if (has_next) {
                         if (has_b) issue_s(1, sn);
+                        ZL_TRACE(0, 7, kv_cnt)
                         if (j + 2 == n_kv) if (mma_lane) mma_commit(&sm.q_empty);  // last S of the item issued
                     }
                 }
@@ -251,7 +268,9 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const int n_kv = (t.kv_len + kTileKV - 1) / kTileKV;
             float m_ref = -INFINITY, l = 0.f;  // reference maximum (raw score units) and row sum
             for (int j = 0; j < n_kv; ++j) {
+                if (quarter == 0) { ZL_TRACE(1 + x, 0, s_cnt) }
                 ZL_WAIT_WARP(&sm.s_full[x], s_cnt & 1, 21);
+                if (quarter == 0) { ZL_TRACE(1 + x, 1, s_cnt) }
                 ++s_cnt;
                 tc_fence_after();
                 float sv[kTileKV];
@@ -263,16 +282,27 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     for (int i = 0; i < 32; ++i) sv[c * 32 + i] = __uint_as_float(r[i]);
                 }
                 tmem_wait_ld();
+                if (quarter == 0) { ZL_TRACE(1 + x, 2, s_cnt - 1) }
                 const int valid = t.kv_len - j * kTileKV;  // columns of this tile inside the task
                 if (valid < kTileKV) {
 #pragma unroll
                     for (int c = 0; c < kTileKV; ++c)
                         if (c >= valid) sv[c] = -INFINITY;  // select, never multiply
                 }
-                float mx = max3(sv[0], sv[1], sv[2]);
+                // four independent chains: a single running maximum is a 64-deep dependent chain
+                float mx0 = max3(sv[0], sv[1], sv[2]), mx1 = max3(sv[3], sv[4], sv[5]);
+                float mx2 = max3(sv[6], sv[7], sv[8]), mx3 = max3(sv[9], sv[10], sv[11]);
 #pragma unroll
-                for (int c = 3; c + 1 < kTileKV; c += 2) mx = max3(mx, sv[c], sv[c + 1]);
-                mx = fmaxf(mx, sv[kTileKV - 1]);
+                for (int c = 12; c + 7 < kTileKV; c += 8) {
+                    mx0 = max3(mx0, sv[c], sv[c + 1]);
+                    mx1 = max3(mx1, sv[c + 2], sv[c + 3]);
+                    mx2 = max3(mx2, sv[c + 4], sv[c + 5]);
+                    mx3 = max3(mx3, sv[c + 6], sv[c + 7]);
+                }
+                // columns 124..127 remain (12 + 8 * 14 = 124)
+                mx0 = max3(mx0, sv[kTileKV - 4], sv[kTileKV - 3]);
+                mx1 = max3(mx1, sv[kTileKV - 2], sv[kTileKV - 1]);
+                const float mx = fmaxf(max3(mx0, mx1, mx2), mx3);
                 // lazy reference update: only when the tile maximum is far above the reference
                 const bool raise = (mx - m_ref) * sl2 > kRescaleThresholdLog2;
                 if (__any_sync(0xffffffffu, raise && j > 0)) {
@@ -293,6 +323,7 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     if (j == 0) l = 0.f;
                     m_ref = mx;
                 }
+                if (quarter == 0) { ZL_TRACE(1 + x, 3, s_cnt - 1) }
                 const float nmb = -m_ref * sl2;
                 float2 sum2 = make_float2(0.f, 0.f);
                 uint32_t pk[kTileKV / 2];
@@ -304,11 +335,14 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     pk[c / 2] = pack_bf16(p0, p1);
                 }
                 l += sum2.x + sum2.y;
+                if (quarter == 0) { ZL_TRACE(1 + x, 4, s_cnt - 1) }
                 tmem_st_x32(lane_addr + col_s, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
                 tmem_st_x32(lane_addr + col_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
                 tmem_wait_st();
+                if (quarter == 0) { ZL_TRACE(1 + x, 5, s_cnt - 1) }
                 tc_fence_before();
                 mbar_arrive(&sm.p_full[x]);
+                if (quarter == 0) { ZL_TRACE(1 + x, 6, s_cnt - 1) }
             }
             // ---- epilogue
             const bool row_ok = row < tile_rows;
