@@ -43,7 +43,7 @@ struct FwdSmem {
     alignas(1024) uint8_t v[kStages][kTileBytes];
     alignas(8) uint64_t q_full[2], q_empty;
     uint64_t kv_full[kStages], kv_empty[kStages];  // K and V of a stage travel together
-    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t s_full[2], p_half[2][2], o_full[2];  // p_half[tile][half of the key columns]
     uint32_t tmem_base;
     volatile int32_t abort_flag;
 };
@@ -112,7 +112,8 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&sm.s_full[x], 1);
-            mbar_init(&sm.p_full[x], 128);
+            mbar_init(&sm.p_half[x][0], 128);
+            mbar_init(&sm.p_half[x][1], 128);
             mbar_init(&sm.o_full[x], 1);
         }
         sm.abort_flag = 0;
@@ -188,10 +189,12 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (mma_lane) mma_commit(&sm.s_full[x]);
             };
             // O_x (+)= P_x V
-            auto issue_pv = [&](int x, uint32_t stage, bool acc) {
+            // (one half of the key columns: P arrives in two halves so that the first four K steps
+            // run while the softmax warps still work on the second half)
+            auto issue_pv = [&](int x, uint32_t stage, bool acc, int half) {
                 const uint64_t dv = dv0 + stage * kTileStep;
 #pragma unroll
-                for (int ks = 0; ks < kTileKV / 16; ++ks)
+                for (int ks = half * (kTileKV / 32); ks < (half + 1) * (kTileKV / 32); ++ks)
                     if (mma_lane) mma_ts(tmem + kColO + x * 128, tmem + kColS + x * 128 + ks * 8, dv + ks * (2048 >> 4), idesc_o,
                            acc || ks > 0);
             };
@@ -219,11 +222,14 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     // tile A: P_A(j) is in TMEM (S_A(j) fully read, O_A rescaled if needed); K(j), V(j)
                     // were waited for when S(j) was issued
                     ZL_TRACE(0, 0, kv_cnt)
-                    ZL_WAIT_WARP(&sm.p_full[0], pa_cnt & 1, 14);
+                    ZL_WAIT_WARP(&sm.p_half[0][0], pa_cnt & 1, 14);
+                    tc_fence_after();
+                    issue_pv(0, s, j > 0, 0);
+                    ZL_WAIT_WARP(&sm.p_half[0][1], pa_cnt & 1, 15);
                     ZL_TRACE(0, 1, kv_cnt)
                     ++pa_cnt;
                     tc_fence_after();
-                    issue_pv(0, s, j > 0);
+                    issue_pv(0, s, true, 1);
                     ZL_TRACE(0, 2, kv_cnt)
                     if (!has_next) if (mma_lane) mma_commit(&sm.o_full[0]);
                     if (has_next) {
@@ -233,11 +239,14 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         ZL_TRACE(0, 4, kv_cnt)
                     }
                     if (has_b) {
-                        ZL_WAIT_WARP(&sm.p_full[1], pb_cnt & 1, 17);
+                        ZL_WAIT_WARP(&sm.p_half[1][0], pb_cnt & 1, 17);
+                        tc_fence_after();
+                        issue_pv(1, s, j > 0, 0);
+                        ZL_WAIT_WARP(&sm.p_half[1][1], pb_cnt & 1, 18);
                         ZL_TRACE(0, 5, kv_cnt)
                         ++pb_cnt;
                         tc_fence_after();
-                        issue_pv(1, s, j > 0);
+                        issue_pv(1, s, true, 1);
                         ZL_TRACE(0, 6, kv_cnt)
                         if (!has_next) if (mma_lane) mma_commit(&sm.o_full[1]);
                     }
@@ -326,22 +335,24 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (quarter == 0) { ZL_TRACE(1 + x, 3, s_cnt - 1) }
                 const float nmb = -m_ref * sl2;
                 float2 sum2 = make_float2(0.f, 0.f);
-                uint32_t pk[kTileKV / 2];
 #pragma unroll
-                for (int c = 0; c < kTileKV; c += 2) {
-                    const float2 e = fma2(make_float2(sv[c], sv[c + 1]), make_float2(sl2, sl2), make_float2(nmb, nmb));
-                    const float p0 = ex2(e.x), p1 = ex2(e.y);
-                    sum2 = add2(sum2, make_float2(p0, p1));
-                    pk[c / 2] = pack_bf16(p0, p1);
+                for (int h = 0; h < 2; ++h) {  // P goes to the MMA warp in two halves of 64 key columns
+                    uint32_t pk[kTileKV / 4];
+#pragma unroll
+                    for (int c = 0; c < kTileKV / 2; c += 2) {
+                        const int cc = h * (kTileKV / 2) + c;
+                        const float2 e = fma2(make_float2(sv[cc], sv[cc + 1]), make_float2(sl2, sl2), make_float2(nmb, nmb));
+                        const float p0 = ex2(e.x), p1 = ex2(e.y);
+                        sum2 = add2(sum2, make_float2(p0, p1));
+                        pk[c / 2] = pack_bf16(p0, p1);
+                    }
+                    tmem_st_x32(lane_addr + col_s + h * 32, pk);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(&sm.p_half[x][h]);
+                    if (quarter == 0) { ZL_TRACE(1 + x, 4 + h, s_cnt - 1) }
                 }
                 l += sum2.x + sum2.y;
-                if (quarter == 0) { ZL_TRACE(1 + x, 4, s_cnt - 1) }
-                tmem_st_x32(lane_addr + col_s, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-                tmem_st_x32(lane_addr + col_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
-                tmem_wait_st();
-                if (quarter == 0) { ZL_TRACE(1 + x, 5, s_cnt - 1) }
-                tc_fence_before();
-                mbar_arrive(&sm.p_full[x]);
                 if (quarter == 0) { ZL_TRACE(1 + x, 6, s_cnt - 1) }
             }
             // ---- epilogue
