@@ -389,7 +389,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const int n_it = count_q_tiles(p, g);
                 ZL_WAIT_WARP(&sm.kv_full, item_cnt & 1, 11);
                 // prologue: S, dP, dV of the item's first query tile and S of the second.
-                // Steady-state order on the tensor pipe: dK(i) dQ(i) dP(i+1) dV(i+1) S(i+2).
+                // Steady-state order on the tensor pipe: dQ(i) dK(i) dP(i+1) dV(i+1) S(i+2).
                 ZL_WAIT_WARP(&sm.q_full[it_cnt & 1], (it_cnt >> 1) & 1, 12);
                 tc_fence_after();
                 issue_s(it_cnt & 1);
@@ -415,16 +415,16 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     {
                         ZL_PROF_SEG_BEGIN
 #pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
+                            if (mma_lane) mma_ss(tmem + kColDP, dds_mn + ks * (2048 >> 4), dk_mn + ks * (2048 >> 4), idesc_dq, ks > 0);
+                        if (mma_lane) mma_commit(&sm.dq_full);  // dQ first: its drain from TMEM runs under the dK MMAs
+                        ZL_TRACE(0, 2, it_cnt)
+#pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
                             const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
                             if (mma_lane) mma_ss(tmem + kColDK, dds_k + off, dq_mn + ks * (2048 >> 4), idesc_dv, i > 0 || ks > 0);
                         }
-                        if (mma_lane) mma_commit(&sm.q_empty[it_cnt & 1]);  // Q stage free early: its reload has dQ, dP, dV to land
-                        ZL_TRACE(0, 2, it_cnt)
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
-                            if (mma_lane) mma_ss(tmem + kColDP, dds_mn + ks * (2048 >> 4), dk_mn + ks * (2048 >> 4), idesc_dq, ks > 0);
-                        if (mma_lane) mma_commit(&sm.dq_full);
+                        if (mma_lane) mma_commit(&sm.q_empty[it_cnt & 1]);
                         if (mma_lane) mma_commit(&sm.ds_free);
                         ZL_PROF_SEG_END(43)
                     }
