@@ -132,6 +132,15 @@ zl_status zl_coalesced_attn_fwd(const zl_tasks* tasks, const void* q, const void
                                 float scale, void* o, float* lse,
                                 float* o_partial, float* lse_partial, void* stream);
 
+/* zl_coalesced_attn_fwd_packed -- the same launch for QKV-packed input (Section IV-D batches Ulysses
+ * sequences through one QKV-packed all-to-all; a fused QKV projection produces the same layout):
+ *   qkv  [T, 3, H, d] bf16, row t = q_t | k_t | v_t.  Needs total_q == total_kv == T (query row i
+ *        and key row i are the same token); ZL_ERR_INVALID_ARG otherwise.
+ * Everything else as zl_coalesced_attn_fwd; results are bit-identical to passing the three
+ * tensors separately (the tiles are fetched through strided tensor maps, nothing is repacked). */
+zl_status zl_coalesced_attn_fwd_packed(const zl_tasks* tasks, const void* qkv, float scale, void* o, float* lse,
+                                       float* o_partial, float* lse_partial, void* stream);
+
 /* zl_lse_merge -- combine the partial results of every merge group (the accumulation step
  * of ring / all-gather context parallelism, Section II-B):
  *     LSE = log sum_t exp(LSE_t),   O = sum_t exp(LSE_t - LSE) * O_t
@@ -157,6 +166,14 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* tasks, const void* q, const void
                                 const void* o, const float* lse, const void* d_o, float scale,
                                 void* dq, void* dk, void* dv,
                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* zl_coalesced_attn_bwd_packed -- the backward for QKV-packed tensors: reads qkv [T, 3, H, d] bf16 and
+ * writes dqkv [T, 3, H, d] bf16 (row t = dq_t | dk_t | dv_t); o, lse, d_o, workspace as above.
+ * Needs total_q == total_kv.  Gradients equal those of zl_coalesced_attn_bwd element for element
+ * (dQ up to the order of the fp32 reduce-adds). */
+zl_status zl_coalesced_attn_bwd_packed(const zl_tasks* tasks, const void* qkv, const void* o, const float* lse,
+                                       const void* d_o, float scale, void* dqkv,
+                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /* zl_coalesced_attn_bwd_noalloc -- the backward for callers that cannot allocate device memory.
  * (The paper has no counterpart; this is a convenience of the library.)

@@ -64,6 +64,10 @@ def _load():
     lib.zl_free_tasks.argtypes = [vp]
     lib.zl_coalesced_attn_fwd.restype = ctypes.c_int
     lib.zl_coalesced_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
+    lib.zl_coalesced_attn_fwd_packed.restype = ctypes.c_int
+    lib.zl_coalesced_attn_fwd_packed.argtypes = [vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
+    lib.zl_coalesced_attn_bwd_packed.restype = ctypes.c_int
+    lib.zl_coalesced_attn_bwd_packed.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
     lib.zl_lse_merge.restype = ctypes.c_int
     lib.zl_lse_merge.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.zl_coalesced_attn_bwd.restype = ctypes.c_int
@@ -223,6 +227,25 @@ def coalesced_attn_bwd(tasks: TaskHandle, q, k, v, o, lse, d_o, scale: float, dq
                                       ctypes.c_float(scale), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
                                       ctypes.c_size_t(workspace_bytes), _stream_ptr(stream)),
            "zl_coalesced_attn_bwd")
+
+
+def coalesced_attn_fwd_packed(tasks: TaskHandle, qkv, scale: float, o, lse, o_partial=None, lse_partial=None,
+                              stream=None):
+    """zl_coalesced_attn_fwd_packed: qkv is [T, 3, H, d] bf16 (total_q == total_kv == T)."""
+    _check(_lib.zl_coalesced_attn_fwd_packed(tasks.ptr, _ptr(qkv), ctypes.c_float(scale), _ptr(o), _ptr(lse),
+                                             _ptr(o_partial), _ptr(lse_partial), _stream_ptr(stream)),
+           "zl_coalesced_attn_fwd_packed")
+
+
+def coalesced_attn_bwd_packed(tasks: TaskHandle, qkv, o, lse, d_o, scale: float, dqkv, workspace,
+                              workspace_bytes: Optional[int] = None, stream=None):
+    """zl_coalesced_attn_bwd_packed: reads qkv [T, 3, H, d], writes dqkv [T, 3, H, d]."""
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(_lib.zl_coalesced_attn_bwd_packed(tasks.ptr, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(d_o),
+                                             ctypes.c_float(scale), _ptr(dqkv), _ptr(workspace),
+                                             ctypes.c_size_t(workspace_bytes), _stream_ptr(stream)),
+           "zl_coalesced_attn_bwd_packed")
 
 
 NOALLOC_SCRATCH_BYTES = 64 * 1024 * 1024

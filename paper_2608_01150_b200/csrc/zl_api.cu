@@ -60,11 +60,13 @@ EncodeTiledFn get_encode_fn() {
 
 // Tensor map over a packed [rows, H, d] bf16 tensor: box = 64 columns x 1 head x box_rows rows,
 // 128-byte swizzle, zero fill outside the tensor.
-bool make_tmap(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim, int box_rows) {
+// `row_stride` (elements) is the distance between token rows: H*d, or 3*H*d for a view into packed QKV.
+bool make_tmap(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim, int box_rows,
+               int64_t row_stride) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)(rows > 0 ? rows : 1)};
-    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)head_dim * 2 * n_heads};
+    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)row_stride * 2};
     cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -265,9 +267,12 @@ void zl_free_tasks(zl_tasks* t) {
     delete t;
 }
 
-zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k, const void* v, float scale,
-                                void* o, float* lse, float* o_partial, float* lse_partial, void* stream) {
-    if (!t) return ZL_ERR_INVALID_ARG;
+}  // extern "C"
+
+namespace {
+// Forward over q, k, v given as token-major views with `in_stride` elements between rows.
+zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* v, int64_t in_stride, float scale,
+                   void* o, float* lse, float* o_partial, float* lse_partial, void* stream) {
     const Schedule& s = t->sched;
     if (s.fwd_items.empty()) return ZL_OK;
     if (t->device < 0) return ZL_ERR_CUDA;
@@ -278,9 +283,9 @@ zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k,
     if (!(scale > 0.f) || !std::isfinite(scale)) return ZL_ERR_INVALID_ARG;
 
     CUtensorMap tq, tk, tv;
-    if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ) ||
-        !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
-        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV))
+    if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ, in_stride) ||
+        !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride) ||
+        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride))
         return ZL_ERR_CUDA;
 
     FwdParams p{};
@@ -330,6 +335,27 @@ zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k,
 #endif
     return ZL_OK;
 }
+}  // namespace
+
+extern "C" {
+
+zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k, const void* v, float scale,
+                                void* o, float* lse, float* o_partial, float* lse_partial, void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    return fwd_impl(t, q, k, v, (int64_t)t->sched.n_heads * t->sched.head_dim, scale, o, lse, o_partial,
+                    lse_partial, stream);
+}
+
+zl_status zl_coalesced_attn_fwd_packed(const zl_tasks* t, const void* qkv, float scale, void* o, float* lse,
+                                       float* o_partial, float* lse_partial, void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    const Schedule& s = t->sched;
+    if (s.total_q != s.total_kv) return ZL_ERR_INVALID_ARG;  // one token row holds its q, k and v
+    if (!qkv) return s.fwd_items.empty() ? ZL_OK : ZL_ERR_INVALID_ARG;
+    const int64_t hd = (int64_t)s.n_heads * s.head_dim;
+    const __nv_bfloat16* base = static_cast<const __nv_bfloat16*>(qkv);
+    return fwd_impl(t, base, base + hd, base + 2 * hd, 3 * hd, scale, o, lse, o_partial, lse_partial, stream);
+}
 
 zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* lse_partial, void* o, float* lse,
                        void* stream) {
@@ -360,10 +386,14 @@ zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* l
     return ZL_OK;
 }
 
-zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k, const void* v, const void* o,
-                                const float* lse, const void* d_o, float scale, void* dq, void* dk, void* dv,
-                                void* workspace, size_t workspace_bytes, void* stream) {
-    if (!t) return ZL_ERR_INVALID_ARG;
+}  // extern "C"
+
+namespace {
+// Backward over q, k, v views with `in_stride` elements between token rows and dq, dk, dv views
+// with `grad_stride` elements between token rows.
+zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* v, int64_t in_stride, const void* o,
+                   const float* lse, const void* d_o, float scale, void* dq, void* dk, void* dv, int64_t grad_stride,
+                   void* workspace, size_t workspace_bytes, void* stream) {
     const Schedule& s = t->sched;
     if (s.tasks.empty()) return ZL_OK;
     if (t->device < 0) return ZL_ERR_CUDA;
@@ -378,10 +408,11 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     CUtensorMap tq, tk, tv, tdo, tdq;
     if (!make_tmap_f32_acc(&tdq, ws + s.ws_dq_acc_off, s.q_pad_total, s.n_heads, s.head_dim)) return ZL_ERR_CUDA;
-    if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ) ||
-        !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
-        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV) ||
-        !make_tmap(&tdo, d_o, s.total_q, s.n_heads, s.head_dim, kTileQ))
+    const int64_t hd = (int64_t)s.n_heads * s.head_dim;
+    if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ, in_stride) ||
+        !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride) ||
+        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride) ||
+        !make_tmap(&tdo, d_o, s.total_q, s.n_heads, s.head_dim, kTileQ, hd))
         return ZL_ERR_CUDA;
 
     BwdParams p{};
@@ -403,6 +434,7 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     p.dq = static_cast<__nv_bfloat16*>(dq);
     p.dk = static_cast<__nv_bfloat16*>(dk);
     p.dv = static_cast<__nv_bfloat16*>(dv);
+    p.grad_row_stride = grad_stride;
     p.dq_acc = reinterpret_cast<float*>(ws + s.ws_dq_acc_off);
     p.aug = ws + s.ws_aug_off;
     p.status = t->d_status;
@@ -458,6 +490,31 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
     }
 #endif
     return ZL_OK;
+}
+}  // namespace
+
+extern "C" {
+
+zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k, const void* v, const void* o,
+                                const float* lse, const void* d_o, float scale, void* dq, void* dk, void* dv,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    const int64_t hd = (int64_t)t->sched.n_heads * t->sched.head_dim;
+    return bwd_impl(t, q, k, v, hd, o, lse, d_o, scale, dq, dk, dv, hd, workspace, workspace_bytes, stream);
+}
+
+zl_status zl_coalesced_attn_bwd_packed(const zl_tasks* t, const void* qkv, const void* o, const float* lse,
+                                       const void* d_o, float scale, void* dqkv, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    const Schedule& s = t->sched;
+    if (s.total_q != s.total_kv) return ZL_ERR_INVALID_ARG;
+    if (!qkv || !dqkv) return s.tasks.empty() ? ZL_OK : ZL_ERR_INVALID_ARG;
+    const int64_t hd = (int64_t)s.n_heads * s.head_dim;
+    const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(qkv);
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(dqkv);
+    return bwd_impl(t, in, in + hd, in + 2 * hd, 3 * hd, o, lse, d_o, scale, out, out + hd, out + 2 * hd, 3 * hd,
+                    workspace, workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(kPreThreads) zl_bwd_post_kernel(const BwdParam
         const int r = slot_row - g.slot;
         if (r >= g.q_len) continue;
         const float* src = p.dq_acc + ((int64_t)slot_row * p.n_heads + h) * D + lane * V;
-        __nv_bfloat16* dst = p.dq + (((int64_t)g.q_off + r) * p.n_heads + h) * D + lane * V;
+        __nv_bfloat16* dst = p.dq + ((int64_t)g.q_off + r) * p.grad_row_stride + h * D + lane * V;
         if constexpr (V == 4) {
             const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
             uint2 o2;
@@ -572,7 +572,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             ZL_WAIT_WARP(&sm.acc_full, item_cnt & 1, 25);
             tc_fence_after();
             const int64_t grow = (int64_t)g.kv_off + wi.row0 + row;
-            __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + (grow * p.n_heads + wi.head) * D;
+            __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + grow * p.grad_row_stride + wi.head * D;
             const float sc = (wg == 0) ? 1.f : p.scale;
             const uint32_t col_acc = (wg == 0) ? kColDV : kColDK;
 #pragma unroll
@@ -598,7 +598,6 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // ------------------------------------------------------------------ dQ warpgroup (one query row per thread)
         reg_inc<152>();
         const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const bool leader = (lane == 0);  // per warp
         uint32_t it_cnt = 0, chunk_cnt = 0;

@@ -58,6 +58,7 @@ struct BwdParams {
     __nv_bfloat16* dq;
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
+    int64_t grad_row_stride;  // elements between token rows of dq, dk, dv (H*d, or 3*H*d when packed)
     float* dq_acc;  // [q_pad_total, H, d]
     uint8_t* aug;   // [H, q_pad_total / 128] tiles of 4 KB: bf16 splits of -lse/scale and -rowsum(dO o O)
     int32_t* status;
