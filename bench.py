@@ -136,7 +136,7 @@ def aggregate_tflops(world: int, flops_per_rank: float, ms_per_step: float) -> f
 class Workload:
     """Device tensors + task handle of one placement."""
 
-    def __init__(self, p, device, seed_shift=0):
+    def __init__(self, p, device, seed_shift=0, flags=0):
         import torch
         import paper_2608_01150_b200 as Z
         import zl_workloads as W
@@ -145,7 +145,7 @@ class Workload:
         mk = lambda rows, s: W.device_normal_bf16((rows, H, d), p.seed * 100 + s + seed_shift, device)
         self.Q, self.K, self.V, self.dO = mk(p.total_q, 0), mk(p.total_kv, 1), mk(p.total_kv, 2), mk(p.total_q, 3)
         t0 = time.perf_counter()
-        self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, H, d)
+        self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, H, d, flags=flags)
         self.build_ms = (time.perf_counter() - t0) * 1e3
         info = self.h.info
         self.O = torch.empty_like(self.Q)
@@ -314,7 +314,7 @@ def run_ours(args):
     peaks, peak_kind = load_peaks()
 
     p = W.config(args.config)
-    wl = Workload(p, device, seed_shift=rank * 7)
+    wl = Workload(p, device, seed_shift=rank * 7, flags=1 if args.fuse_local_chunks else 0)
     K, Wm = args.steps, max(3, args.warmup)
     for _ in range(Wm):
         wl.step()
@@ -380,6 +380,7 @@ def run_ours(args):
         "config": {"workload": p.name, "n_heads": p.n_heads, "head_dim": p.head_dim, "total_q": p.total_q,
                    "total_kv": p.total_kv, "tasks": int(wl.h.info.n_tasks),
                    "step": "fwd launch + lse merge + bwd (pre, main, post)",
+                   "fuse_local_chunks": bool(args.fuse_local_chunks),
                    "l2": "inputs larger than L2 (K+V alone exceed 126 MB); no flush",
                    "parallelism": f"{world} independent rank-local placements"},
         "fwd_tflops": aggregate_tflops(world, p.fwd_flops(), ms_fwd / K),
@@ -418,6 +419,24 @@ def run_ours(args):
             except Exception as e:  # noqa: BLE001
                 extra[f"cfg{ci}"] = {"error": repr(e)}
         result["per_config"] = extra
+        if not args.fuse_local_chunks and p.shards:
+            # the same workload with ZL_BUILD_FUSE_LOCAL_CHUNKS (one final task per query range whose chunks are
+            # contiguous: no partials, nothing to merge) -- reported beside the headline, never instead of it
+            try:
+                wf = Workload(p, device, flags=1)
+                for _ in range(3):
+                    wf.step()
+                tf = wf.time_region(wf.fwd, 5) / 5
+                ts = wf.time_region(wf.step, 5) / 5
+                result["fused_local_chunks"] = {
+                    "value": (p.fwd_flops() + p.bwd_flops()) / ts / 1e9, "unit": "TFLOP/s", "ms_per_step": ts,
+                    "fwd_ms": tf, "fwd_tflops": p.fwd_flops() / tf / 1e9,
+                    "fused_ranges": int(wf.h.info.n_fused_ranges), "tasks": int(wf.h.info.n_tasks),
+                    "note": "optional schedule (bench.py --fuse-local-chunks); the headline value keeps the merge step"}
+                del wf
+                torch.cuda.empty_cache()
+            except Exception as e:  # noqa: BLE001
+                result["fused_local_chunks"] = {"error": repr(e)}
 
     if world == 1 and rank == 0 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(p)
@@ -514,6 +533,9 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="named configuration 1..5 (default: Wan-14B-shaped rank)")
     ap.add_argument("--extra-configs", default="2,3,5", help="also time these configurations (N=1 only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fuse-local-chunks", action="store_true",
+                    help="build the handle with ZL_BUILD_FUSE_LOCAL_CHUNKS: query ranges whose chunks are contiguous run "
+                         "as one final task (no partials, nothing to merge); off by default")
     ap.add_argument("--ablation", default="", choices=["", "straggler", "coalescing"],
                     help="print an extra measurement instead of the benchmark line")
     args = ap.parse_args()

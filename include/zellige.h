@@ -67,6 +67,7 @@ typedef struct {
     size_t o_partial_bytes;     /* partial_rows * n_heads * head_dim * 4 */
     size_t lse_partial_bytes;   /* n_heads * partial_rows * 4 */
     size_t bwd_workspace_bytes; /* scratch needed by zl_coalesced_attn_bwd */
+    int32_t n_fused_ranges; /* shard query ranges lowered to one final task (zl_build_tasks_ex) */
 } zl_tasks_info;
 
 /* zl_build_tasks -- lower a placement into the rank-local schedule (Section IV-D: "lowers
@@ -95,6 +96,24 @@ zl_status zl_build_tasks(const int32_t* cu_seqlens, int32_t n_whole,
                          const zl_shard_desc* shards, int32_t n_shards,
                          int32_t total_q, int32_t total_kv, int32_t n_heads, int32_t head_dim,
                          void* stream, zl_tasks** out);
+
+/* zl_build_tasks_ex -- zl_build_tasks with options (flags = 0 is zl_build_tasks).
+ *
+ * ZL_BUILD_FUSE_LOCAL_CHUNKS: a shard query range whose non-empty key chunks are all on this rank
+ * and, sorted by offset, tile one contiguous interval of KV-space is lowered to ONE task over
+ * that interval instead of one task per chunk.  It is exact attention over the union (the same
+ * result the merge produces, Section II-B), final after the forward launch: such a range has no
+ * partial slots (zl_tasks_get_partial_slot reports rows_padded = 0 for its shards), is not a
+ * merge group, and its backward work units are the tiles of the whole interval.  Fusion is applied
+ * to every such range or to none: it is skipped when a fused interval would partially overlap
+ * another key range of the placement (e.g. another query range that uses only some of the
+ * chunks).  The paper's engine has no counterpart: it receives remote chunks over a ring or an
+ * all-gather; this is the case where the all-gather has already made them contiguous. */
+#define ZL_BUILD_FUSE_LOCAL_CHUNKS 1u
+zl_status zl_build_tasks_ex(const int32_t* cu_seqlens, int32_t n_whole,
+                            const zl_shard_desc* shards, int32_t n_shards,
+                            int32_t total_q, int32_t total_kv, int32_t n_heads, int32_t head_dim,
+                            uint32_t flags, void* stream, zl_tasks** out);
 
 zl_status zl_tasks_get_info(const zl_tasks* tasks, zl_tasks_info* info);
 

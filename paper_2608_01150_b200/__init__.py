@@ -8,5 +8,5 @@ kernels.  PyTorch is used for device memory and streams.  There is no CPU fallba
 from .binding import (ZlError, TaskHandle, ShardDesc, TasksInfo, build_tasks,  # noqa: F401
                       coalesced_attn_fwd, lse_merge, coalesced_attn_bwd, coalesced_attn_bwd_noalloc,
                       coalesced_attn_fwd_packed, coalesced_attn_bwd_packed,
-                      NOALLOC_SCRATCH_BYTES, launch_count,
+                      NOALLOC_SCRATCH_BYTES, BUILD_FUSE_LOCAL_CHUNKS, launch_count,
                       library_path, STATUS_NAMES)

@@ -37,7 +37,7 @@ class TasksInfo(ctypes.Structure):
                 ("n_kv_groups", ctypes.c_int32), ("n_fwd_items", ctypes.c_int32),
                 ("n_bwd_items", ctypes.c_int32), ("partial_rows", ctypes.c_int64),
                 ("o_partial_bytes", ctypes.c_size_t), ("lse_partial_bytes", ctypes.c_size_t),
-                ("bwd_workspace_bytes", ctypes.c_size_t)]
+                ("bwd_workspace_bytes", ctypes.c_size_t), ("n_fused_ranges", ctypes.c_int32)]
 
 
 def library_path() -> str:
@@ -53,6 +53,8 @@ def _load():
     vp, i32, i64p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64)
     lib.zl_build_tasks.restype = ctypes.c_int
     lib.zl_build_tasks.argtypes = [vp, i32, vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+    lib.zl_build_tasks_ex.restype = ctypes.c_int
+    lib.zl_build_tasks_ex.argtypes = [vp, i32, vp, i32, i32, i32, i32, i32, ctypes.c_uint32, vp, ctypes.POINTER(vp)]
     lib.zl_tasks_get_info.restype = ctypes.c_int
     lib.zl_tasks_get_info.argtypes = [vp, ctypes.POINTER(TasksInfo)]
     lib.zl_tasks_get_partial_slot.restype = ctypes.c_int
@@ -190,16 +192,25 @@ class TaskHandle:
             pass
 
 
+BUILD_FUSE_LOCAL_CHUNKS = 1
+
+
 def build_tasks(cu_seqlens: Sequence[int], shards: Sequence[Sequence[int]], total_q: int, total_kv: int,
-                n_heads: int, head_dim: int, stream=None) -> TaskHandle:
-    """zl_build_tasks: placement (cu_seqlens + shard descriptors) -> task handle."""
+                n_heads: int, head_dim: int, stream=None, flags: int = 0) -> TaskHandle:
+    """zl_build_tasks / zl_build_tasks_ex: placement (cu_seqlens + shard descriptors) -> task handle.
+    flags: 0 or BUILD_FUSE_LOCAL_CHUNKS."""
     n_whole = max(0, len(cu_seqlens) - 1)
     cu = (ctypes.c_int32 * max(1, len(cu_seqlens)))(*[int(c) for c in cu_seqlens])
     sh = (ShardDesc * max(1, len(shards)))(*[ShardDesc(*[int(v) for v in s]) for s in shards])
     out = ctypes.c_void_p()
-    st = _lib.zl_build_tasks(ctypes.cast(cu, ctypes.c_void_p) if len(cu_seqlens) else None, n_whole,
-                             ctypes.cast(sh, ctypes.c_void_p) if len(shards) else None, len(shards),
-                             total_q, total_kv, n_heads, head_dim, _stream_ptr(stream), ctypes.byref(out))
+    cu_p = ctypes.cast(cu, ctypes.c_void_p) if len(cu_seqlens) else None
+    sh_p = ctypes.cast(sh, ctypes.c_void_p) if len(shards) else None
+    if flags:
+        st = _lib.zl_build_tasks_ex(cu_p, n_whole, sh_p, len(shards), total_q, total_kv, n_heads, head_dim,
+                                    ctypes.c_uint32(flags), _stream_ptr(stream), ctypes.byref(out))
+    else:
+        st = _lib.zl_build_tasks(cu_p, n_whole, sh_p, len(shards), total_q, total_kv, n_heads, head_dim,
+                                 _stream_ptr(stream), ctypes.byref(out))
     _check(st, "zl_build_tasks")
     return TaskHandle(out.value, n_heads, head_dim, total_q, total_kv, len(shards))
 

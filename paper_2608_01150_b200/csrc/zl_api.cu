@@ -145,12 +145,20 @@ int64_t zl_launch_count(void) { return g_launches.load(); }
 zl_status zl_build_tasks(const int32_t* cu_seqlens, int32_t n_whole, const zl_shard_desc* shards,
                          int32_t n_shards, int32_t total_q, int32_t total_kv, int32_t n_heads,
                          int32_t head_dim, void* stream, zl_tasks** out) {
+    return zl_build_tasks_ex(cu_seqlens, n_whole, shards, n_shards, total_q, total_kv, n_heads, head_dim, 0u,
+                             stream, out);
+}
+
+zl_status zl_build_tasks_ex(const int32_t* cu_seqlens, int32_t n_whole, const zl_shard_desc* shards,
+                            int32_t n_shards, int32_t total_q, int32_t total_kv, int32_t n_heads,
+                            int32_t head_dim, uint32_t flags, void* stream, zl_tasks** out) {
     if (!out) return ZL_ERR_INVALID_ARG;
     *out = nullptr;
+    if (flags & ~ZL_BUILD_FUSE_LOCAL_CHUNKS) return ZL_ERR_INVALID_ARG;
     zl_tasks* h = new (std::nothrow) zl_tasks();
     if (!h) return ZL_ERR_INVALID_ARG;
     zl_status st = build_schedule(cu_seqlens, n_whole, shards, n_shards, total_q, total_kv, n_heads, head_dim,
-                                  &h->sched);
+                                  flags, &h->sched);
     if (st != ZL_OK) { delete h; return st; }
 
     int n_dev = 0;
@@ -223,6 +231,7 @@ zl_status zl_tasks_get_info(const zl_tasks* t, zl_tasks_info* info) {
     info->n_kv_groups = (int32_t)s.kv_groups.size();
     info->n_fwd_items = (int32_t)s.fwd_items.size();
     info->n_bwd_items = (int32_t)s.bwd_items.size();
+    info->n_fused_ranges = s.n_fused_ranges;
     info->partial_rows = s.partial_rows;
     info->o_partial_bytes = (size_t)s.partial_rows * s.n_heads * s.head_dim * sizeof(float);
     info->lse_partial_bytes = (size_t)s.partial_rows * s.n_heads * sizeof(float);

@@ -58,15 +58,17 @@ struct Schedule {
     std::vector<WorkItem> fwd_items;
     std::vector<WorkItem> bwd_items;
     int64_t partial_rows = 0;
+    int32_t n_fused_ranges = 0;             // shard query ranges lowered to one final task (chunk fusion)
     size_t bwd_workspace_bytes = 0;
     // byte offsets inside the backward workspace
     size_t ws_dq_acc_off = 0, ws_aug_off = 0;
 };
 
 // Validates the placement and fills `s`.  Pure host code, no CUDA.
+// `flags`: ZL_BUILD_* bits of zl_build_tasks_ex.
 zl_status build_schedule(const int32_t* cu_seqlens, int32_t n_whole, const zl_shard_desc* shards,
                          int32_t n_shards, int32_t total_q, int32_t total_kv, int32_t n_heads,
-                         int32_t head_dim, Schedule* s);
+                         int32_t head_dim, uint32_t flags, Schedule* s);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -36,7 +36,7 @@ bool identical_or_disjoint(std::vector<Range> r) {
 
 zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc* shards,
                          int32_t n_shards, int32_t total_q, int32_t total_kv, int32_t n_heads,
-                         int32_t head_dim, Schedule* s) {
+                         int32_t head_dim, uint32_t flags, Schedule* s) {
     if (!s || n_whole < 0 || n_shards < 0 || total_q < 0 || total_kv < 0 || n_heads <= 0)
         return ZL_ERR_INVALID_ARG;
     if ((n_whole > 0 && !cu) || (n_shards > 0 && !shards)) return ZL_ERR_INVALID_ARG;
@@ -66,6 +66,44 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
         q_ranges.push_back({cu[i], len});
         kv_ranges.push_back({cu[i], len});
     }
+    // Optional fusion of local chunks: a query range whose non-empty key chunks, sorted by offset,
+    // tile one contiguous interval needs no partials and no merge -- it is exact attention over
+    // the interval, i.e. one task that is final after the forward launch.  Done for all such
+    // ranges or for none: the fused intervals must still be identical-or-disjoint with every other
+    // key range of the placement.
+    std::vector<int32_t> fuse_leader(n_shards, -1);  // per shard: first shard of its fused range, or -1
+    std::vector<Range> fuse_union(n_shards, Range{0, 0});
+    if ((flags & ZL_BUILD_FUSE_LOCAL_CHUNKS) && n_shards > 0) {
+        std::map<std::pair<int64_t, int64_t>, std::vector<int32_t>> by_q;
+        bool sane = true;
+        for (int i = 0; i < n_shards && sane; ++i) {
+            const zl_shard_desc& d = shards[i];
+            if (d.q_len < 0 || d.kv_len < 0 || d.q_off < 0 || d.kv_off < 0) sane = false;
+            else if (d.q_len > 0) by_q[{d.q_off, d.q_len}].push_back(i);
+        }
+        std::vector<Range> all_kv;
+        for (int i = 0; i < n_whole; ++i)
+            if (cu[i + 1] > cu[i]) all_kv.push_back({cu[i], cu[i + 1] - cu[i]});
+        for (auto& kvp : by_q) {
+            if (!sane) break;
+            std::vector<Range> chunks;
+            for (int32_t i : kvp.second)
+                if (shards[i].kv_len > 0) chunks.push_back({shards[i].kv_off, shards[i].kv_len});
+            std::sort(chunks.begin(), chunks.end());
+            bool contiguous = chunks.size() >= 2;
+            for (size_t c = 1; c < chunks.size() && contiguous; ++c)
+                contiguous = chunks[c - 1].off + chunks[c - 1].len == chunks[c].off;
+            if (contiguous) {
+                const Range u{chunks.front().off, chunks.back().off + chunks.back().len - chunks.front().off};
+                for (int32_t i : kvp.second) { fuse_leader[i] = kvp.second.front(); fuse_union[i] = u; }
+                all_kv.push_back(u);
+            } else {
+                for (const Range& c : chunks) all_kv.push_back(c);
+            }
+        }
+        if (!sane || !identical_or_disjoint(all_kv)) std::fill(fuse_leader.begin(), fuse_leader.end(), -1);
+    }
+
     // shards
     s->shard_to_task.assign(n_shards, -1);
     s->shard_slot_off.assign(n_shards, 0);
@@ -92,6 +130,22 @@ zl_status build_schedule(const int32_t* cu, int32_t n_whole, const zl_shard_desc
         Task t{};
         t.q_off = d.q_off; t.q_len = d.q_len; t.kv_off = d.kv_off; t.kv_len = d.kv_len;
         t.kv_group = -1; t.q_group = -1; t.q_slot = 0;
+        if (fuse_leader[i] >= 0) {
+            // fused query range: its first shard carries the task over the whole interval, final
+            // after the forward launch; the other shards of the range add nothing
+            if (d.kv_len > 0) kv_ranges.back() = fuse_union[i];
+            if (fuse_leader[i] != i) {
+                if (shards[fuse_leader[i]].seq_id != d.seq_id) return ZL_ERR_INVALID_ARG;
+                s->shard_to_task[i] = s->shard_to_task[fuse_leader[i]];
+                continue;
+            }
+            t.kv_off = (int32_t)fuse_union[i].off; t.kv_len = (int32_t)fuse_union[i].len;
+            t.partial_slot = -1;
+            s->shard_to_task[i] = (int32_t)s->tasks.size();
+            s->tasks.push_back(t);
+            ++s->n_fused_ranges;
+            continue;
+        }
         auto mk = std::make_pair((int64_t)d.q_off, (int64_t)d.q_len);
         auto it = merge_index.find(mk);
         if (it == merge_index.end()) {

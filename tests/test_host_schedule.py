@@ -139,3 +139,63 @@ def test_launch_without_device_fails_loudly(Z):
     with pytest.raises(Z.ZlError) as e:
         Z.coalesced_attn_fwd(h, 16, 16, 16, 0.125, 16, 16, 16, 16, stream=0)
     assert e.value.status == 5      # ZL_ERR_CUDA: no fallback path exists
+
+
+# ---------------------------------------------------------------- fusion of local chunks (zl_build_tasks_ex)
+def _build_fused(Z, p):
+    return Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, p.n_heads, p.head_dim,
+                         flags=Z.BUILD_FUSE_LOCAL_CHUNKS)
+
+
+def test_fusion_lowers_contiguous_chunks_to_one_final_task(Z):
+    # one image of 100 rows; query range A = [100,300) over three chunks given out of order that tile
+    # [100,700); query range B = [300,500) over the same three chunks
+    shards = [(100, 200, 300, 200, 0), (100, 200, 100, 200, 0), (100, 200, 500, 200, 0),
+              (300, 200, 100, 200, 1), (300, 200, 300, 200, 1), (300, 200, 500, 200, 1)]
+    p = W.custom_placement("fuse", 2, 64, 0, [0, 100], shards, 500, 700)
+    plain, fused = _build(Z, p), _build_fused(Z, p)
+    assert (plain.info.n_tasks, plain.info.n_merge_groups, plain.info.n_fused_ranges) == (7, 2, 0)
+    assert plain.info.partial_rows == 6 * 256
+    assert (fused.info.n_tasks, fused.info.n_merge_groups, fused.info.n_fused_ranges) == (3, 0, 2)
+    assert fused.info.partial_rows == 0 and fused.info.n_kv_groups == 2    # the image and [100,700)
+    assert all(fused.partial_slot(i) == (0, 0) for i in range(len(shards)))
+    # forward items: every query row of the 3 tasks once per head; key length 600 sorts first
+    items = fused.fwd_items()
+    assert sorted({t for (t, _, _, _) in items}) == [0, 1, 2]
+    rows = {}
+    for (t, hd, r0, n) in items:
+        rows[(t, hd)] = rows.get((t, hd), 0) + n
+    assert sorted(rows.values()) == sorted([100, 100, 200, 200, 200, 200])
+    # backward: the interval's 600 key rows once per head, plus the image's 100
+    got = {}
+    for (g, hd, r0, n) in fused.bwd_items():
+        got[(g, hd)] = got.get((g, hd), 0) + n
+    assert sorted(got.values()) == [100, 100, 600, 600]
+
+
+def test_fusion_is_all_or_nothing(Z):
+    # range B uses only two of A's three chunks: fusing A would partially overlap B's chunks -> no fusion at all
+    shards = [(0, 64, 0, 100, 0), (0, 64, 100, 100, 0), (0, 64, 200, 100, 0),
+              (64, 64, 0, 100, 1), (64, 64, 100, 100, 1)]
+    p = W.custom_placement("nofuse", 1, 64, 0, [0], shards, 128, 300)
+    plain, fused = _build(Z, p), _build_fused(Z, p)
+    assert fused.info.n_fused_ranges == 0
+    assert (fused.info.n_tasks, fused.info.n_merge_groups, fused.info.partial_rows) == \
+           (plain.info.n_tasks, plain.info.n_merge_groups, plain.info.partial_rows)
+    assert fused.fwd_items() == plain.fwd_items() and fused.bwd_items() == plain.bwd_items()
+
+
+def test_fusion_needs_contiguous_chunks_and_keeps_validation(Z):
+    # a gap between the chunks: not fused; a single chunk: nothing to fuse
+    p = W.custom_placement("gap", 1, 64, 0, [0], [(0, 64, 0, 100, 0), (0, 64, 150, 100, 0), (64, 10, 300, 20, 1)], 80, 320)
+    h = _build_fused(Z, p)
+    assert h.info.n_fused_ranges == 0 and h.info.n_merge_groups == 2
+    # invalid input is still rejected with the same status
+    bad = W.custom_placement("bad", 1, 64, 0, [0], [(0, 64, 0, 100, 0), (0, 64, 0, 100, 0)], 64, 100)
+    for flags in (0, Z.BUILD_FUSE_LOCAL_CHUNKS):
+        with pytest.raises(Z.ZlError) as e:
+            Z.build_tasks(bad.cu_seqlens, bad.shards, bad.total_q, bad.total_kv, 1, 64, flags=flags)
+        assert e.value.status == 2       # ZL_ERR_OVERLAP: duplicate (query range, key range)
+    with pytest.raises(Z.ZlError) as e:
+        Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, 1, 64, flags=2)
+    assert e.value.status == 1           # unknown flag

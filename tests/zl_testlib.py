@@ -40,12 +40,12 @@ def dev_to_f64(t: torch.Tensor) -> np.ndarray:
 class GpuRun:
     """Runs forward (+merge) and optionally backward for a placement through the binding."""
 
-    def __init__(self, p, scale=None):
+    def __init__(self, p, scale=None, flags=0):
         import paper_2608_01150_b200 as Z
         self.Z = Z
         self.p = p
         self.scale = p.scale if scale is None else scale
-        self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, p.n_heads, p.head_dim)
+        self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, p.n_heads, p.head_dim, flags=flags)
         self.info = self.h.info
 
     def forward(self, Q, K, V, merge=True):
