@@ -415,13 +415,15 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    CUtensorMap tq, tk, tv, tdo, tdq;
+    CUtensorMap tq, tk, tv, tdo, tdq, tdk, tdv;
     if (!make_tmap_f32_acc(&tdq, ws + s.ws_dq_acc_off, s.q_pad_total, s.n_heads, s.head_dim)) return ZL_ERR_CUDA;
     const int64_t hd = (int64_t)s.n_heads * s.head_dim;
     if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ, in_stride) ||
         !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride) ||
         !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride) ||
-        !make_tmap(&tdo, d_o, s.total_q, s.n_heads, s.head_dim, kTileQ, hd))
+        !make_tmap(&tdo, d_o, s.total_q, s.n_heads, s.head_dim, kTileQ, hd) ||
+        !make_tmap(&tdk, dk, s.total_kv, s.n_heads, s.head_dim, kTileKV, grad_stride) ||
+        !make_tmap(&tdv, dv, s.total_kv, s.n_heads, s.head_dim, kTileKV, grad_stride))
         return ZL_ERR_CUDA;
 
     BwdParams p{};
@@ -466,7 +468,7 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     if (p.n_items > 0) {
         const int grid = std::min<int>(t->n_sms, p.n_items);
         LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
-        if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, tdq, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
+        if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, tdq, tdk, tdv, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
         g_launches.fetch_add(1);
     }
     {

@@ -229,7 +229,8 @@ template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                   const __grid_constant__ CUtensorMap tm_dq, const BwdParams p) {
+                   const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_dk,
+                   const __grid_constant__ CUtensorMap tm_dv, const BwdParams p) {
     using Smem = BwdSmem<D>;
     constexpr int kBoxes = Smem::kBoxes;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -269,6 +270,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         prefetch_tmap(&tm_v);
         prefetch_tmap(&tm_do);
         prefetch_tmap(&tm_dq);
+        prefetch_tmap(&tm_dk);
+        prefetch_tmap(&tm_dv);
     }
     // constant A operand of the augmentation steps: 128 rows x 8 bf16 per block
     for (int i = threadIdx.x; i < 3 * 2048 / 4; i += kBwdThreads) {
@@ -467,6 +470,8 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t ds_row_addr = smem_u32(sm.ds) + row * 128;
         const float sl2 = p.scale_log2;
         uint32_t item_cnt = 0, it_cnt = 0;
+        const bool store_leader = (warp & 3) == 0 && lane == 0;  // one thread per warpgroup issues its TMA stores
+        bool store_pending = false;
         for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
             const WorkItem wi = p.items[it];
             const KvGroup g = p.kv_groups[wi.unit];
@@ -524,6 +529,12 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ZL_WAIT_WARP(&sm.dp_full, it_cnt & 1, 23);
                     if (warp == 4 && lane == 0) { ZL_TRACE(1, 3, it_cnt) }
                     if (it_cnt > 0) ZL_WAIT_WARP(&sm.ds_free, (it_cnt - 1) & 1, 24);  // dS buffer consumed by dK/dQ
+                    if (store_pending) {
+                        // this warpgroup's box of the dS tile staged the previous item's dK / dV tile
+                        if (store_leader) bulk_wait_group_read<0>();
+                        named_bar_sync(2 + wg, 128);
+                        store_pending = false;
+                    }
                     if (warp == 4 && lane == 0) { ZL_TRACE(1, 4, it_cnt) }
                     tc_fence_after();
                     {
@@ -571,29 +582,67 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // ---- epilogue: warpgroup 0 stores dV, warpgroup 1 stores dK (scaled)
             ZL_WAIT_WARP(&sm.acc_full, item_cnt & 1, 25);
             tc_fence_after();
-            const int64_t grow = (int64_t)g.kv_off + wi.row0 + row;
-            __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + grow * p.grad_row_stride + wi.head * D;
             const float sc = (wg == 0) ? 1.f : p.scale;
             const uint32_t col_acc = (wg == 0) ? kColDV : kColDK;
+            if (wi.rows == kTileKV) {
+                // full key tile: stage 64 columns at a time in this warpgroup's box of the (now idle) dS
+                // tile and write them with one TMA store each -- coalesced, and the warpgroup moves on to
+                // the next item while the copy engine drains the box
+                const uint32_t box_addr = smem_u32(sm.ds) + wg * Smem::kBoxBytes + row * 128;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_x32(lane_addr + col_acc + c * 32, r);
-                tmem_wait_ld();
-                if (row_ok) {
+                for (int b = 0; b < kBoxes; ++b) {
+                    if (b > 0) {
+                        if (store_leader) bulk_wait_group_read<0>();
+                        named_bar_sync(2 + wg, 128);
+                    }
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 o4;
-                        o4.x = pack_bf16(__uint_as_float(r[i]) * sc, __uint_as_float(r[i + 1]) * sc);
-                        o4.y = pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc);
-                        o4.z = pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc);
-                        o4.w = pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc);
-                        *reinterpret_cast<uint4*>(dst + c * 32 + i) = o4;
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_x32(lane_addr + col_acc + b * 64 + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            const int i = k4 * 8;
+                            st_shared_v4(box_addr + (((c * 4 + k4) ^ (row & 7)) << 4),
+                                         pack_bf16(__uint_as_float(r[i]) * sc, __uint_as_float(r[i + 1]) * sc),
+                                         pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc),
+                                         pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc),
+                                         pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc));
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    named_bar_sync(2 + wg, 128);
+                    if (store_leader) {
+                        tma_store_3d(wg == 0 ? &tm_dv : &tm_dk, sm.ds + wg * Smem::kBoxBytes, b * 64, wi.head,
+                                     g.kv_off + wi.row0);
+                        bulk_commit_group();
+                    }
+                }
+                store_pending = true;
+            } else {
+                const int64_t grow = (int64_t)g.kv_off + wi.row0 + row;
+                __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + grow * p.grad_row_stride + wi.head * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_x32(lane_addr + col_acc + c * 32, r);
+                    tmem_wait_ld();
+                    if (row_ok) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8) {
+                            uint4 o4;
+                            o4.x = pack_bf16(__uint_as_float(r[i]) * sc, __uint_as_float(r[i + 1]) * sc);
+                            o4.y = pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc);
+                            o4.z = pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc);
+                            o4.w = pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + i) = o4;
+                        }
                     }
                 }
             }
             tc_fence_before();
         }
+        if (store_leader) bulk_wait_group<0>();  // the last dK / dV stores have left shared memory and landed
     } else {
         // ------------------------------------------------------------------ dQ warpgroup (one query row per thread)
         reg_inc<152>();
@@ -670,8 +719,8 @@ teardown:
 
 template <int D>
 cudaError_t launch_main_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                          const CUtensorMap& tdo, const CUtensorMap& tdq, const BwdParams& p, int grid,
-                          cudaStream_t stream) {
+                          const CUtensorMap& tdo, const CUtensorMap& tdq, const CUtensorMap& tdk,
+                          const CUtensorMap& tdv, const BwdParams& p, int grid, cudaStream_t stream) {
     constexpr int smem = sizeof(BwdSmem<D>);
     static bool configured = false;
     if (!configured) {
@@ -679,7 +728,7 @@ cudaError_t launch_main_t(const CUtensorMap& tq, const CUtensorMap& tk, const CU
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    zl_bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, tdq, p);
+    zl_bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, tdq, tdk, tdv, p);
     return cudaGetLastError();
 }
 
@@ -694,11 +743,11 @@ cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStre
 }
 
 cudaError_t launch_bwd_main(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                            const CUtensorMap& tdo, const CUtensorMap& tdq, const BwdParams& p, int grid,
-                            cudaStream_t stream) {
+                            const CUtensorMap& tdo, const CUtensorMap& tdq, const CUtensorMap& tdk,
+                            const CUtensorMap& tdv, const BwdParams& p, int grid, cudaStream_t stream) {
     if (p.n_items == 0) return cudaSuccess;
-    return head_dim == 128 ? launch_main_t<128>(tq, tk, tv, tdo, tdq, p, grid, stream)
-                           : launch_main_t<64>(tq, tk, tv, tdo, tdq, p, grid, stream);
+    return head_dim == 128 ? launch_main_t<128>(tq, tk, tv, tdo, tdq, tdk, tdv, p, grid, stream)
+                           : launch_main_t<64>(tq, tk, tv, tdo, tdq, tdk, tdv, p, grid, stream);
 }
 
 cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream) {

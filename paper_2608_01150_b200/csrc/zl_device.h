@@ -67,8 +67,8 @@ struct BwdParams {
 
 cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
 cudaError_t launch_bwd_main(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                            const CUtensorMap& tdo, const CUtensorMap& tdq, const BwdParams& p, int grid,
-                            cudaStream_t stream);
+                            const CUtensorMap& tdo, const CUtensorMap& tdq, const CUtensorMap& tdk,
+                            const CUtensorMap& tdv, const BwdParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
 
 cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
