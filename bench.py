@@ -38,7 +38,7 @@ METRIC = "coalesced attention TFLOP/s fwd and fwd+bwd; % of B200 dense BF16 peak
 # DRAM traffic of the backward main kernel from one ncu capture on configuration 3
 # (dram__bytes_read.sum + dram__bytes_write.sum, profiles/zl_bwd_main_kernel_cfg3.txt); scaled to the
 # benchmarked workload by the counted backward FLOPs, which the K/V and Q/dO streaming follows.
-NCU_BWD_MAIN_CFG3_DRAM_BYTES = 2.457673e9 + 1.442899e9
+NCU_BWD_MAIN_CFG3_DRAM_BYTES = 2.647806e9 + 1.529451e9
 NCU_BWD_MAIN_CFG3_FLOPS = 2.5 * 4.0 * (16 * 1560 * 1560 + 8 * 8190 * 8190) * 128 * 12
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
