@@ -16,7 +16,7 @@ namespace {
 constexpr int kMergeThreads = 256;
 
 template <int D>
-__global__ void __launch_bounds__(kMergeThreads) zl_merge_kernel(const MergeParams p) {
+__global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeParams p) {  // 8 blocks = 64 warps per SM
     constexpr int V = D / 32;  // floats per lane: 4 (d=128) or 2 (d=64)
     const int lane = threadIdx.x & 31;
     const int warps_per_block = kMergeThreads / 32;
