@@ -58,46 +58,63 @@ __device__ __forceinline__ void split3(float x, __nv_bfloat16 (&h)[3]) {
 // end of the query range get -1e30 and 0, which makes their P and dS vanish.
 template <int D>
 __global__ void __launch_bounds__(kPreThreads) zl_bwd_pre_kernel(const BwdParams p) {
-    constexpr int V = D / 32;
+    // One warp per (8 consecutive padded query rows, head): four lanes share a row, each reading a
+    // quarter of its O and dO (16-byte loads), so a warp keeps 4 KB (d=128) in flight and the two
+    // 16-byte halves of the eight rows land in the augmentation tile as two contiguous 128-byte stores.
+    constexpr int kPerLane = D / 4;  // bf16 elements of one row handled by one lane
     const int lane = threadIdx.x & 31;
-    const int64_t n_units = (int64_t)p.q_pad_total * p.n_heads;
+    const int sub = lane >> 2, quarter = lane & 3;
+    const int64_t n_units = (int64_t)(p.q_pad_total / 8) * p.n_heads;
     const float inv_scale = 1.f / p.scale;
     for (int64_t u = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); u < n_units;
          u += (int64_t)gridDim.x * (kPreThreads / 32)) {
-        const int slot_row = (int)(u / p.n_heads);
-        const int h = (int)(u - (int64_t)slot_row * p.n_heads);
-        const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, slot_row)];
+        const int row8 = (int)(u / p.n_heads);
+        const int h = (int)(u - (int64_t)row8 * p.n_heads);
+        const int slot_row = row8 * 8 + sub;
+        // slots are padded to 128 rows: the eight rows belong to one query group
+        const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, row8 * 8)];
         const int r = slot_row - g.slot;
         float xd = 0.f, xl = -1e30f;
-        if (r < g.q_len) {
+        const bool live = r < g.q_len;
+        float acc = 0.f;
+        if (live) {
             const int64_t row = (int64_t)g.q_off + r;
-            const __nv_bfloat16* po = p.o + (row * p.n_heads + h) * D + lane * V;
-            const __nv_bfloat16* pd = p.d_o + (row * p.n_heads + h) * D + lane * V;
-            float acc = 0.f;
+            const uint4* po = reinterpret_cast<const uint4*>(p.o + (row * p.n_heads + h) * D + quarter * kPerLane);
+            const uint4* pd = reinterpret_cast<const uint4*>(p.d_o + (row * p.n_heads + h) * D + quarter * kPerLane);
+            uint4 a[kPerLane / 8], b[kPerLane / 8];
 #pragma unroll
-            for (int i = 0; i < V; i += 2) {
-                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + i));
-                const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pd + i));
-                acc = fmaf(a.x, b.x, acc);
-                acc = fmaf(a.y, b.y, acc);
+            for (int i = 0; i < kPerLane / 8; ++i) { a[i] = __ldg(po + i); b[i] = __ldg(pd + i); }
+#pragma unroll
+            for (int i = 0; i < kPerLane / 8; ++i) {
+                const uint32_t aw[4] = {a[i].x, a[i].y, a[i].z, a[i].w}, bw[4] = {b[i].x, b[i].y, b[i].z, b[i].w};
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[w]));
+                    const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[w]));
+                    acc = fmaf(fa.x, fb.x, acc);
+                    acc = fmaf(fa.y, fb.y, acc);
+                }
             }
-#pragma unroll
-            for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+        }
+        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+        if (live) {
             xd = -acc;
-            const float l = p.lse[(int64_t)h * p.total_q + row];
+            const float l = p.lse[(int64_t)h * p.total_q + (int64_t)g.q_off + r];
             if (l > -INFINITY && l < INFINITY) xl = -l * inv_scale;
         }
-        // lanes 0..15 write the 16 bf16 elements of this row (32 bytes in two 16-byte halves)
-        if (lane < 16) {
-            __nv_bfloat16 hl[3], hd[3];
-            split3(xl, hl);
-            split3(xd, hd);
-            __nv_bfloat16 val = __float2bfloat16_rn(0.f);
-            if (lane < 3) val = hl[lane];
-            else if (lane >= 8 && lane < 11) val = hd[lane - 8];
+        // lane quarter 0 writes elements 0..7 of its row (-LSE/scale pieces), quarter 1 elements 8..15 (-D pieces)
+        if (quarter < 2) {
+            __nv_bfloat16 hp[3];
+            split3(quarter == 0 ? xl : xd, hp);
+            uint4 val;
+            val.x = (uint32_t)__bfloat16_as_ushort(hp[0]) | ((uint32_t)__bfloat16_as_ushort(hp[1]) << 16);
+            val.y = (uint32_t)__bfloat16_as_ushort(hp[2]);
+            val.z = 0u;
+            val.w = 0u;
             const int tile = slot_row / kTileQ, tr = slot_row % kTileQ;
             uint8_t* base = p.aug + ((int64_t)h * (p.q_pad_total / kTileQ) + tile) * 4096;
-            *reinterpret_cast<__nv_bfloat16*>(base + (lane / 8) * 2048 + (tr / 8) * 128 + (tr % 8) * 16 + (lane % 8) * 2) = val;
+            *reinterpret_cast<uint4*>(base + quarter * 2048 + (tr / 8) * 128 + (tr % 8) * 16) = val;
         }
     }
 }
