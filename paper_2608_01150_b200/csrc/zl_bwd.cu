@@ -122,27 +122,42 @@ __global__ void __launch_bounds__(kPreThreads) zl_bwd_pre_kernel(const BwdParams
 // ======================================================================= post
 template <int D>
 __global__ void __launch_bounds__(kPreThreads) zl_bwd_post_kernel(const BwdParams p) {
+    // One warp per padded query row: every head of the row in batches of four, all four 16-byte loads
+    // of a batch issued before the first conversion (2 KB in flight per warp at d=128).
     constexpr int V = D / 32;
+    constexpr int kBatch = 4;
     const int lane = threadIdx.x & 31;
-    const int64_t n_units = (int64_t)p.q_pad_total * p.n_heads;
-    for (int64_t u = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); u < n_units;
-         u += (int64_t)gridDim.x * (kPreThreads / 32)) {
-        const int slot_row = (int)(u / p.n_heads);
-        const int h = (int)(u - (int64_t)slot_row * p.n_heads);
-        const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, slot_row)];
-        const int r = slot_row - g.slot;
+    for (int64_t slot_row = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); slot_row < p.q_pad_total;
+         slot_row += (int64_t)gridDim.x * (kPreThreads / 32)) {
+        const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, (int)slot_row)];
+        const int r = (int)slot_row - g.slot;
         if (r >= g.q_len) continue;
-        const float* src = p.dq_acc + ((int64_t)slot_row * p.n_heads + h) * D + lane * V;
-        __nv_bfloat16* dst = p.dq + ((int64_t)g.q_off + r) * p.grad_row_stride + h * D + lane * V;
-        if constexpr (V == 4) {
-            const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
-            uint2 o2;
-            o2.x = pack_bf16(x.x * p.scale, x.y * p.scale);
-            o2.y = pack_bf16(x.z * p.scale, x.w * p.scale);
-            *reinterpret_cast<uint2*>(dst) = o2;
-        } else {
-            const float2 x = __ldcs(reinterpret_cast<const float2*>(src));
-            *reinterpret_cast<uint32_t*>(dst) = pack_bf16(x.x * p.scale, x.y * p.scale);
+        const float* src = p.dq_acc + slot_row * p.n_heads * D + lane * V;
+        __nv_bfloat16* dst = p.dq + ((int64_t)g.q_off + r) * p.grad_row_stride + lane * V;
+        for (int h0 = 0; h0 < p.n_heads; h0 += kBatch) {
+            if constexpr (V == 4) {
+                float4 x[kBatch];
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i)
+                    if (h0 + i < p.n_heads) x[i] = __ldcs(reinterpret_cast<const float4*>(src + (int64_t)(h0 + i) * D));
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i)
+                    if (h0 + i < p.n_heads) {
+                        uint2 o2;
+                        o2.x = pack_bf16(x[i].x * p.scale, x[i].y * p.scale);
+                        o2.y = pack_bf16(x[i].z * p.scale, x[i].w * p.scale);
+                        *reinterpret_cast<uint2*>(dst + (int64_t)(h0 + i) * D) = o2;
+                    }
+            } else {
+                float2 x[kBatch];
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i)
+                    if (h0 + i < p.n_heads) x[i] = __ldcs(reinterpret_cast<const float2*>(src + (int64_t)(h0 + i) * D));
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i)
+                    if (h0 + i < p.n_heads)
+                        *reinterpret_cast<uint32_t*>(dst + (int64_t)(h0 + i) * D) = pack_bf16(x[i].x * p.scale, x[i].y * p.scale);
+            }
         }
     }
 }
