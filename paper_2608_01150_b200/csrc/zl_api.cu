@@ -100,12 +100,12 @@ struct LaunchTimer {
 };
 
 // Tensor map over the fp32 dQ accumulator [rows, H, d]: box = 32 columns x 1 head x 128 rows.
-bool make_tmap_f32_acc(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim) {
+bool make_tmap_f32_acc(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim, int box_rows = 32) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)(rows > 0 ? rows : 1)};
     cuuint64_t strides[2] = {(cuuint64_t)head_dim * 4, (cuuint64_t)head_dim * 4 * n_heads};
-    cuuint32_t box[3] = {32, 1, 32};  // one warp's 32 query rows x 32 fp32 columns
+    cuuint32_t box[3] = {32, 1, (cuuint32_t)box_rows};  // 32 fp32 columns x one warp's 32 rows (dQ) or a 128-row tile
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -291,10 +291,16 @@ zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
         return ZL_ERR_INVALID_ARG;
     if (!(scale > 0.f) || !std::isfinite(scale)) return ZL_ERR_INVALID_ARG;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to, top;
+    const int64_t hd = (int64_t)s.n_heads * s.head_dim;
     if (!make_tmap(&tq, q, s.total_q, s.n_heads, s.head_dim, kTileQ, in_stride) ||
         !make_tmap(&tk, k, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride) ||
-        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride))
+        !make_tmap(&tv, v, s.total_kv, s.n_heads, s.head_dim, kTileKV, in_stride) ||
+        !make_tmap(&to, o, s.total_q, s.n_heads, s.head_dim, kTileQ, hd))
+        return ZL_ERR_CUDA;
+    // partial results leave through the same kind of store; without shards the map is never used
+    if (s.partial_rows > 0 ? !make_tmap_f32_acc(&top, o_partial, s.partial_rows, s.n_heads, s.head_dim, kTileQ)
+                           : !make_tmap(&top, o, s.total_q, s.n_heads, s.head_dim, kTileQ, hd))
         return ZL_ERR_CUDA;
 
     FwdParams p{};
@@ -321,7 +327,7 @@ zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     const int grid = std::min<int>(t->n_sms, p.n_items);
     {
         LaunchTimer lt(t, ZL_K_FWD, static_cast<cudaStream_t>(stream));
-        if (launch_fwd(s.head_dim, tq, tk, tv, p, grid, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        if (launch_fwd(s.head_dim, tq, tk, tv, to, top, p, grid, static_cast<cudaStream_t>(stream)) != cudaSuccess)
             return ZL_ERR_CUDA;
     }
     g_launches.fetch_add(1);

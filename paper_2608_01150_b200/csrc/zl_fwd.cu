@@ -41,6 +41,7 @@ struct FwdSmem {
     alignas(1024) uint8_t q[2][kTileBytes];
     alignas(1024) uint8_t k[kStages][kTileBytes];
     alignas(1024) uint8_t v[kStages][kTileBytes];
+    alignas(1024) uint8_t o_stage[2][kBoxBytes];  // per softmax warpgroup: 128 rows x 128 bytes of O on their way out
     alignas(8) uint64_t q_full[2], q_empty;
     uint64_t kv_full[kStages], kv_empty[kStages];  // K and V of a stage travel together
     uint64_t s_full[2], p_half[2][2], o_full[2];  // p_half[tile][half of the key columns]
@@ -84,7 +85,8 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-              const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
+              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+              const __grid_constant__ CUtensorMap tm_op, const FwdParams p) {
     using Smem = FwdSmem<D>;
     constexpr int kStages = Smem::kStages;
     constexpr int kBoxes = Smem::kBoxes;
@@ -121,6 +123,8 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         prefetch_tmap(&tm_q);
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
+        prefetch_tmap(&tm_o);
+        prefetch_tmap(&tm_op);
     }
     if (warp == 1) {
         tmem_alloc(&sm.tmem_base, kTmemCols);
@@ -268,6 +272,8 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const uint32_t col_s = kColS + x * 128, col_o = kColO + x * 128;
         uint32_t s_cnt = 0, o_cnt = 0;
+        const bool store_leader = quarter == 0 && lane == 0;  // one thread per warpgroup issues its TMA stores
+        bool store_pending = false;                            // this warpgroup's box may still be read by a store
         const float sl2 = p.scale_log2;
         for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
             const WorkItem wi = p.items[it];
@@ -364,8 +370,71 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 ++o_cnt;
                 tc_fence_after();
             }
-            const int64_t grow = (int64_t)(t.partial_slot >= 0 ? t.partial_slot : t.q_off) + wi.row0 + x * kTileQ + row;
-            if (t.partial_slot >= 0) {
+            const int64_t grow0 = (int64_t)(t.partial_slot >= 0 ? t.partial_slot : t.q_off) + wi.row0 + x * kTileQ;
+            const int64_t grow = grow0 + row;
+            if (tile_rows == kTileQ && n_kv > 0) {
+                // full tile: stage 128 bytes per row at a time in this warpgroup's box and write each box
+                // with one TMA store -- coalesced, and the warpgroup is free for the next item while the
+                // copy engine drains the box
+                const uint32_t box_row = smem_u32(sm.o_stage[x]) + row * 128;
+                if (t.partial_slot >= 0) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {  // 32 fp32 columns per box
+                        if (c > 0 || store_pending) {
+                            if (store_leader) bulk_wait_group_read<0>();
+                            named_bar_sync(2 + x, 128);
+                        }
+                        uint32_t r[32];
+                        tmem_ld_x32(lane_addr + col_o + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k4 = 0; k4 < 8; ++k4)
+                            st_shared_v4(box_row + ((k4 ^ (row & 7)) << 4),
+                                         __float_as_uint(__uint_as_float(r[k4 * 4]) * inv_l),
+                                         __float_as_uint(__uint_as_float(r[k4 * 4 + 1]) * inv_l),
+                                         __float_as_uint(__uint_as_float(r[k4 * 4 + 2]) * inv_l),
+                                         __float_as_uint(__uint_as_float(r[k4 * 4 + 3]) * inv_l));
+                        fence_proxy_async_smem();
+                        named_bar_sync(2 + x, 128);
+                        if (store_leader) {
+                            tma_store_3d(&tm_op, sm.o_stage[x], c * 32, wi.head, (int32_t)grow0);
+                            bulk_commit_group();
+                        }
+                    }
+                    p.lse_partial[(int64_t)wi.head * p.partial_rows + grow] = lse;
+                } else {
+#pragma unroll
+                    for (int b = 0; b < D / 64; ++b) {  // 64 bf16 columns per box
+                        if (b > 0 || store_pending) {
+                            if (store_leader) bulk_wait_group_read<0>();
+                            named_bar_sync(2 + x, 128);
+                        }
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t r[32];
+                            tmem_ld_x32(lane_addr + col_o + b * 64 + c * 32, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4) {
+                                const int i = k4 * 8;
+                                st_shared_v4(box_row + (((c * 4 + k4) ^ (row & 7)) << 4),
+                                             pack_bf16(__uint_as_float(r[i]) * inv_l, __uint_as_float(r[i + 1]) * inv_l),
+                                             pack_bf16(__uint_as_float(r[i + 2]) * inv_l, __uint_as_float(r[i + 3]) * inv_l),
+                                             pack_bf16(__uint_as_float(r[i + 4]) * inv_l, __uint_as_float(r[i + 5]) * inv_l),
+                                             pack_bf16(__uint_as_float(r[i + 6]) * inv_l, __uint_as_float(r[i + 7]) * inv_l));
+                            }
+                        }
+                        fence_proxy_async_smem();
+                        named_bar_sync(2 + x, 128);
+                        if (store_leader) {
+                            tma_store_3d(&tm_o, sm.o_stage[x], b * 64, wi.head, (int32_t)grow0);
+                            bulk_commit_group();
+                        }
+                    }
+                    p.lse[(int64_t)wi.head * p.total_q + grow] = lse;
+                }
+                store_pending = true;
+            } else if (t.partial_slot >= 0) {
                 float* dst = p.o_partial + (grow * p.n_heads + wi.head) * D;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
@@ -415,6 +484,7 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
             tc_fence_before();
         }
+        if (store_leader) bulk_wait_group<0>();  // the last O stores have left shared memory and landed
     }
 
 teardown:
@@ -428,8 +498,8 @@ teardown:
 }
 
 template <int D>
-cudaError_t launch_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                     int grid, cudaStream_t stream) {
+cudaError_t launch_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                     const CUtensorMap& top, const FwdParams& p, int grid, cudaStream_t stream) {
     constexpr int smem = sizeof(FwdSmem<D>);
     static bool configured = false;
     if (!configured) {
@@ -437,16 +507,18 @@ cudaError_t launch_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    zl_fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, p);
+    zl_fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, to, top, p);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                       const FwdParams& p, int grid, cudaStream_t stream) {
+                       const CUtensorMap& to, const CUtensorMap& top, const FwdParams& p, int grid,
+                       cudaStream_t stream) {
     if (p.n_items == 0) return cudaSuccess;
-    return head_dim == 128 ? launch_t<128>(tq, tk, tv, p, grid, stream) : launch_t<64>(tq, tk, tv, p, grid, stream);
+    return head_dim == 128 ? launch_t<128>(tq, tk, tv, to, top, p, grid, stream)
+                           : launch_t<64>(tq, tk, tv, to, top, p, grid, stream);
 }
 
 }  // namespace zl
