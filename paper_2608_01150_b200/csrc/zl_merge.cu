@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeP
         for (int t = 0; t < g.n_parts; ++t) {
             const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
             const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
-            z += (M == -INFINITY) ? 0.f : expf(lt - M);
+            z += (M == -INFINITY) ? 0.f : __expf(lt - M);
         }
         const float L = (M == -INFINITY) ? -INFINITY : M + logf(z);
         float acc[V];
@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeP
         for (int t = 0; t < g.n_parts; ++t) {
             const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
             const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
-            const float w = (L == -INFINITY) ? 0.f : expf(lt - L);
+            const float w = (L == -INFINITY) ? 0.f : __expf(lt - L);
             const float* src = p.o_partial + (pr * p.n_heads + h) * D + lane * V;
             if constexpr (V == 4) {
                 const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
