@@ -132,6 +132,13 @@ zl_status zl_tasks_get_bwd_items(const zl_tasks* tasks, int32_t* items, int32_t 
 
 void zl_free_tasks(zl_tasks* tasks);
 
+/* Stream behaviour of the compute entry points (zl_coalesced_attn_fwd / _fwd_packed, zl_lse_merge,
+ * zl_coalesced_attn_bwd / _bwd_packed): each only enqueues kernels (and, for the backward, one memset)
+ * on `stream`; tensor maps are encoded on the host at call time and passed by value.  They do not
+ * synchronise, so a whole step can be captured in a CUDA graph and replayed (the captured tensor
+ * addresses are baked in); make the first call on a handle's device outside the capture.
+ * zl_last_device_status, zl_get_kernel_timing and enabled kernel timing are not capturable. */
+
 /* zl_coalesced_attn_fwd -- one persistent launch over the whole work list (Section IV-D:
  * whole sequences packed into one block-diagonal attention call, shards run beside them).
  *
