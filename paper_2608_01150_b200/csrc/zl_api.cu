@@ -392,9 +392,11 @@ zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* l
     p.lse_partial = lse_partial;
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
+    int max_parts = 0;
+    for (const MergeGroup& mg : s.merge_groups) max_parts = std::max(max_parts, (int)mg.n_parts);
     {
         LaunchTimer lt(t, ZL_K_MERGE, static_cast<cudaStream_t>(stream));
-        if (launch_merge(s.head_dim, p, t->n_sms, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        if (launch_merge(s.head_dim, p, max_parts, t->n_sms, static_cast<cudaStream_t>(stream)) != cudaSuccess)
             return ZL_ERR_CUDA;
     }
     g_launches.fetch_add(1);

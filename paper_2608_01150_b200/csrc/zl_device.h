@@ -74,7 +74,8 @@ cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStr
 cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                        const CUtensorMap& to, const CUtensorMap& top, const FwdParams& p, int grid,
                        cudaStream_t stream);
-cudaError_t launch_merge(int head_dim, const MergeParams& p, int n_sms, cudaStream_t stream);
+// `max_parts`: the largest number of parts of any merge group (selects a register-resident variant).
+cudaError_t launch_merge(int head_dim, const MergeParams& p, int max_parts, int n_sms, cudaStream_t stream);
 cudaError_t launch_wait_selftest(int32_t* status, uint64_t limit_ns, cudaStream_t stream);
 
 }  // namespace zl

@@ -15,7 +15,47 @@ namespace {
 
 constexpr int kMergeThreads = 256;
 
-template <int D>
+// Up to NP parts: the parts' LSEs are read once and kept in registers (weights e_t / z).
+template <int D, int NP>
+__device__ __forceinline__ float merge_small(const MergeParams& p, const MergeGroup& g, int row, int h, int lane,
+                                             float (&acc)[D / 32]) {
+    constexpr int V = D / 32;
+    const float* lse_h = p.lse_partial + (int64_t)h * p.partial_rows + row;
+    const int32_t* part = p.parts + g.part_begin;
+    float lt[NP];
+    float M = -INFINITY;
+#pragma unroll
+    for (int t = 0; t < NP; ++t) {
+        lt[t] = (t < g.n_parts) ? __ldg(lse_h + part[t]) : -INFINITY;
+        M = fmaxf(M, lt[t]);
+    }
+    float z = 0.f;
+#pragma unroll
+    for (int t = 0; t < NP; ++t) {
+        lt[t] = (M == -INFINITY) ? 0.f : __expf(lt[t] - M);  // 0 for absent parts
+        z += lt[t];
+    }
+    const float inv_z = (z > 0.f) ? 1.f / z : 0.f;
+#pragma unroll
+    for (int t = 0; t < NP; ++t) {
+        if (t < g.n_parts) {
+            const float w = lt[t] * inv_z;
+            const float* src = p.o_partial + (((int64_t)part[t] + row) * p.n_heads + h) * D + lane * V;
+            if constexpr (V == 4) {
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
+                acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+                acc[2] = fmaf(w, x.z, acc[2]); acc[3] = fmaf(w, x.w, acc[3]);
+            } else {
+                const float2 x = __ldcs(reinterpret_cast<const float2*>(src));
+                acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+            }
+        }
+    }
+    return (M == -INFINITY) ? -INFINITY : M + logf(z);
+}
+
+// NP = 4 or 8: every group has at most NP parts (chosen by the launcher); NP = 0: any number of parts.
+template <int D, int NP>
 __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeParams p) {  // 8 blocks = 64 warps per SM
     constexpr int V = D / 32;  // floats per lane: 4 (d=128) or 2 (d=64)
     const int lane = threadIdx.x & 31;
@@ -34,33 +74,39 @@ __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeP
         }
         const MergeGroup g = p.groups[lo];
         const int row = (int)(r - p.row_prefix[lo]);
-        float M = -INFINITY;
-        for (int t = 0; t < g.n_parts; ++t) {
-            const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
-            M = fmaxf(M, __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr));
-        }
-        float z = 0.f;
-        for (int t = 0; t < g.n_parts; ++t) {
-            const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
-            const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
-            z += (M == -INFINITY) ? 0.f : __expf(lt - M);
-        }
-        const float L = (M == -INFINITY) ? -INFINITY : M + logf(z);
         float acc[V];
 #pragma unroll
         for (int i = 0; i < V; ++i) acc[i] = 0.f;
-        for (int t = 0; t < g.n_parts; ++t) {
-            const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
-            const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
-            const float w = (L == -INFINITY) ? 0.f : __expf(lt - L);
-            const float* src = p.o_partial + (pr * p.n_heads + h) * D + lane * V;
-            if constexpr (V == 4) {
-                const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
-                acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
-                acc[2] = fmaf(w, x.z, acc[2]); acc[3] = fmaf(w, x.w, acc[3]);
-            } else {
-                const float2 x = __ldcs(reinterpret_cast<const float2*>(src));
-                acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+        float L;
+        if constexpr (NP > 0) {
+            L = merge_small<D, NP>(p, g, row, h, lane, acc);
+        } else {
+            // any number of parts: three passes over the parts' LSEs
+            float M = -INFINITY;
+            for (int t = 0; t < g.n_parts; ++t) {
+                const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
+                M = fmaxf(M, __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr));
+            }
+            float z = 0.f;
+            for (int t = 0; t < g.n_parts; ++t) {
+                const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
+                const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
+                z += (M == -INFINITY) ? 0.f : __expf(lt - M);
+            }
+            L = (M == -INFINITY) ? -INFINITY : M + logf(z);
+            for (int t = 0; t < g.n_parts; ++t) {
+                const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
+                const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
+                const float w = (L == -INFINITY) ? 0.f : __expf(lt - L);
+                const float* src = p.o_partial + (pr * p.n_heads + h) * D + lane * V;
+                if constexpr (V == 4) {
+                    const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
+                    acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+                    acc[2] = fmaf(w, x.z, acc[2]); acc[3] = fmaf(w, x.w, acc[3]);
+                } else {
+                    const float2 x = __ldcs(reinterpret_cast<const float2*>(src));
+                    acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+                }
             }
         }
         const int64_t qrow = (int64_t)g.q_off + row;
@@ -81,13 +127,19 @@ __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeP
 
 }  // namespace
 
-cudaError_t launch_merge(int head_dim, const MergeParams& p, int n_sms, cudaStream_t stream) {
+cudaError_t launch_merge(int head_dim, const MergeParams& p, int max_parts, int n_sms, cudaStream_t stream) {
     if (p.n_groups == 0) return cudaSuccess;
     const int grid = n_sms * 8;  // 8 resident blocks of 256 threads per SM
-    if (head_dim == 128)
-        zl_merge_kernel<128><<<grid, kMergeThreads, 0, stream>>>(p);
-    else
-        zl_merge_kernel<64><<<grid, kMergeThreads, 0, stream>>>(p);
+    const int np = max_parts <= 4 ? 4 : (max_parts <= 8 ? 8 : 0);
+    if (head_dim == 128) {
+        if (np == 4) zl_merge_kernel<128, 4><<<grid, kMergeThreads, 0, stream>>>(p);
+        else if (np == 8) zl_merge_kernel<128, 8><<<grid, kMergeThreads, 0, stream>>>(p);
+        else zl_merge_kernel<128, 0><<<grid, kMergeThreads, 0, stream>>>(p);
+    } else {
+        if (np == 4) zl_merge_kernel<64, 4><<<grid, kMergeThreads, 0, stream>>>(p);
+        else if (np == 8) zl_merge_kernel<64, 8><<<grid, kMergeThreads, 0, stream>>>(p);
+        else zl_merge_kernel<64, 0><<<grid, kMergeThreads, 0, stream>>>(p);
+    }
     return cudaGetLastError();
 }
 
