@@ -352,6 +352,25 @@ def run_ours(args):
                 "frac_of_burst": (achieved / float(peaks.get("bf16_tflops", 1590.0)) if achieved else None),
                 "traffic": NCU_BWD_MAIN_CFG3_DRAM_BYTES * p.bwd_flops() / NCU_BWD_MAIN_CFG3_FLOPS,
                 "traffic_note": "bytes per launch, scaled by counted FLOPs from an ncu capture on configuration 3"}
+    # The same kernel against shared-memory bandwidth (128 B/clk/SM), which is what actually binds the one-CTA
+    # formulation: bytes through shared memory per (128-row query tile, 128-row key tile, head) -- MMA operand
+    # reads, TMA tile writes, dS stores, dQ staging writes and the reduce engine's reads of them.
+    d = p.head_dim
+    b_mn = 16 * d * 2                                   # B operand of one K step when N = d
+    per_pair = (2 * ((d // 16) * 8192 + 8192)           # S^T and dP^T: A + B per K step, plus the augmentation step
+                + 8 * b_mn + 2 * 8 * (4096 + b_mn)      # dV (A from TMEM), dK, dQ
+                + 2 * 128 * d * 2 + 4096                # TMA writes of Q, dO and the augmentation tile
+                + 128 * 128 * 2                         # dS^T tile written by the P/dS warps
+                + 2 * 128 * d * 4)                      # dQ staged in fp32 and read back by the reduce
+    tasks_qk = [(l, l) for l in p.whole_lengths()] + [(s[1], s[3]) for s in p.shards]
+    n_pairs = p.n_heads * sum(-(-q // 128) * -(-k // 128) for q, k in tasks_qk)
+    n_sms = torch.cuda.get_device_properties(device).multi_processor_count
+    sm_hz = float(clocks.get("sm_mhz") or 0.0) * 1e6
+    if bm and sm_hz:
+        b_clk = per_pair * n_pairs / (n_sms * bm * 1e-3 * sm_hz)
+        roofline["smem"] = {"bytes_per_tile_pair": per_pair, "tile_pairs": n_pairs, "achieved": b_clk, "peak": 128.0,
+                            "unit": "B/clk/SM", "frac": b_clk / 128.0,
+                            "note": "shared-memory traffic of the same launches over the sampled median SM clock"}
     fm = kernels["fwd"]["avg_ms"]
     fwd_kernel_tflops = p.fwd_flops() / (fm * 1e-3) / 1e12 if fm else None
     mm = kernels["merge"]["avg_ms"]
