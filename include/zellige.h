@@ -27,6 +27,14 @@
  *   - Outputs land at the input token offsets whatever the internal work order
  *     (Section IV-D: outputs keep the rank-local input order).
  *   - A handle may be in flight on one stream at a time.
+ *   - A handle belongs to the device that was current when it was built; every compute entry
+ *     point returns ZL_ERR_INVALID_ARG when another device is current.
+ *   - Every element of Q, K, V and d_o inside [0, total_q) / [0, total_kv) must be finite,
+ *     including rows that no task covers: a ragged last tile is fetched as a whole 128-row
+ *     tile, the rows beyond the task are masked by selection (their scores, P and dS become
+ *     exactly -inf / 0), but their values still enter the tensor-core products, where
+ *     0 * Inf or 0 * NaN would poison the valid rows of that tile.  Finite neighbours of any
+ *     magnitude cannot leak.
  */
 #ifndef ZELLIGE_H_
 #define ZELLIGE_H_
@@ -219,7 +227,9 @@ zl_status zl_coalesced_attn_bwd_packed(const zl_tasks* tasks, const void* qkv, c
  *     handle must have been built beforehand (zl_build_tasks allocates its small tables), and
  *     kernel timing must be off on the handle (ZL_ERR_INVALID_ARG otherwise: timing creates events).
  *   - The first call on each device looks up the device address of the scratch array; make that
- *     first call outside any stream capture.
+ *     first call outside any stream capture.  The first launch of each kernel on a device may also
+ *     load its code, so a caller that needs a strictly allocation-free region should have run one
+ *     backward (this entry point or zl_coalesced_attn_bwd) on the device before entering it.
  *   - All calls on a device share the one array and it keeps whatever the last call left in it.
  *     The part that must start at zero (the dQ accumulator) is cleared on the stream by every
  *     call.  Two calls that overlap on the GPU (different streams, or different handles at the

@@ -33,10 +33,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-I", os.path.join(_ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    if os.environ.get("ZL_PROFILE_BUILD"):
-        cmd += ["-DZL_PROFILE"]
-        if os.environ["ZL_PROFILE_BUILD"] == "trace":  # event timestamps only, no per-site counters
-            cmd += ["-DZL_TRACE_ONLY"]
     cmd += ["-o", LIB + ".tmp"] + _sources()
     subprocess.run(cmd, check=True)
     os.replace(LIB + ".tmp", LIB)

@@ -115,6 +115,12 @@ bool make_tmap_f32_acc(CUtensorMap* m, const void* base, int64_t rows, int n_hea
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Launches go to the current device: it has to be the one the handle's tables live on.
+bool on_handle_device(const zl_tasks* t) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == t->device;
+}
+
 template <class T>
 size_t place(size_t& off, size_t count) {
     off = align_up(off, 256);
@@ -285,6 +291,7 @@ zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     const Schedule& s = t->sched;
     if (s.fwd_items.empty()) return ZL_OK;
     if (t->device < 0) return ZL_ERR_CUDA;
+    if (!on_handle_device(t)) return ZL_ERR_INVALID_ARG;
     if (!q || !k || !v || !o || !lse) return ZL_ERR_INVALID_ARG;
     if (s.partial_rows > 0 && (!o_partial || !lse_partial)) return ZL_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(o_partial))
@@ -316,14 +323,6 @@ zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     p.o_partial = o_partial;
     p.lse_partial = lse_partial;
     p.status = t->d_status;
-#ifdef ZL_PROFILE
-    static long long* d_fprof = nullptr;
-    if (getenv("ZL_PROF")) {
-        if (!d_fprof) cudaMalloc(&d_fprof, 1024 * sizeof(long long));
-        cudaMemsetAsync(d_fprof, 0, 1024 * sizeof(long long), static_cast<cudaStream_t>(stream));
-        p.prof = d_fprof;
-    }
-#endif
     const int grid = std::min<int>(t->n_sms, p.n_items);
     {
         LaunchTimer lt(t, ZL_K_FWD, static_cast<cudaStream_t>(stream));
@@ -331,23 +330,6 @@ zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
             return ZL_ERR_CUDA;
     }
     g_launches.fetch_add(1);
-#ifdef ZL_PROFILE
-    if (p.prof && getenv("ZL_TRACE")) {
-        long long hprof[1024];
-        cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
-        cudaMemcpy(hprof, p.prof, sizeof(hprof), cudaMemcpyDeviceToHost);
-        const long long t0 = hprof[256 + 0];
-        for (int role = 0; role < 3; ++role)
-            for (int itx = 0; itx < 8; ++itx) {
-                fprintf(stderr, "[zl fwd trace] role %d it %d:", role, 200 + itx);
-                for (int ev = 0; ev < 11; ++ev) {
-                    const long long v = hprof[256 + role * 128 + itx * 16 + ev];
-                    if (v) fprintf(stderr, " e%d=%lld", ev, v - t0);
-                }
-                fprintf(stderr, "\n");
-            }
-    }
-#endif
     return ZL_OK;
 }
 }  // namespace
@@ -378,6 +360,7 @@ zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* l
     const Schedule& s = t->sched;
     if (s.merge_groups.empty()) return ZL_OK;
     if (t->device < 0) return ZL_ERR_CUDA;
+    if (!on_handle_device(t)) return ZL_ERR_INVALID_ARG;
     if (!o_partial || !lse_partial || !o || !lse) return ZL_ERR_INVALID_ARG;
     if (!aligned16(o_partial) || !aligned16(o)) return ZL_ERR_INVALID_ARG;
     MergeParams p{};
@@ -414,6 +397,7 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     const Schedule& s = t->sched;
     if (s.tasks.empty()) return ZL_OK;
     if (t->device < 0) return ZL_ERR_CUDA;
+    if (!on_handle_device(t)) return ZL_ERR_INVALID_ARG;
     if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !workspace) return ZL_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
@@ -458,14 +442,6 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     p.aug = ws + s.ws_aug_off;
     p.status = t->d_status;
 
-#ifdef ZL_PROFILE
-    static long long* d_prof = nullptr;
-    if (getenv("ZL_PROF")) {
-        if (!d_prof) cudaMalloc(&d_prof, 1024 * sizeof(long long));
-        cudaMemsetAsync(d_prof, 0, 1024 * sizeof(long long), cs);
-        p.prof = d_prof;
-    }
-#endif
     if (cudaMemsetAsync(p.dq_acc, 0, (size_t)s.q_pad_total * s.n_heads * s.head_dim * sizeof(float), cs) != cudaSuccess)
         return ZL_ERR_CUDA;
     {
@@ -484,30 +460,6 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
         if (launch_bwd_post(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
     }
     g_launches.fetch_add(1);
-#ifdef ZL_PROFILE
-    if (p.prof) {
-        long long hprof[1024];
-        cudaStreamSynchronize(cs);
-        cudaMemcpy(hprof, p.prof, sizeof(hprof), cudaMemcpyDeviceToHost);
-        for (int b = 0; b < 2; ++b) {
-            fprintf(stderr, "[zl prof] cta %d total %lld :", b, hprof[b * 64]);
-            for (int i = 1; i < 64; ++i) if (hprof[b * 64 + i]) fprintf(stderr, " s%d=%lld", i, hprof[b * 64 + i]);
-            fprintf(stderr, "\n");
-        }
-        if (getenv("ZL_TRACE")) {
-            const long long t0 = hprof[256 + 0];
-            for (int role = 0; role < 3; ++role)
-                for (int itx = 0; itx < 8; ++itx) {
-                    fprintf(stderr, "[zl trace] role %d it %d:", role, 200 + itx);
-                    for (int ev = 0; ev < 11; ++ev) {
-                        const long long v = hprof[256 + role * 128 + itx * 16 + ev];
-                        if (v) fprintf(stderr, " e%d=%lld", ev, v - t0);
-                    }
-                    fprintf(stderr, "\n");
-                }
-        }
-    }
-#endif
     return ZL_OK;
 }
 }  // namespace
@@ -569,9 +521,8 @@ zl_status zl_coalesced_attn_bwd_noalloc(const zl_tasks* t, const void* q, const 
     if (t->device < 0) return ZL_ERR_CUDA;
     if (t->timing) return ZL_ERR_INVALID_ARG;  // per-kernel timing creates events: not allocation-free
     if (t->sched.bwd_workspace_bytes > (size_t)ZL_NOALLOC_SCRATCH_BYTES) return ZL_ERR_WORKSPACE;
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev != t->device) return ZL_ERR_CUDA;
-    void* scratch = noalloc_scratch_for(dev);
+    if (!on_handle_device(t)) return ZL_ERR_INVALID_ARG;
+    void* scratch = noalloc_scratch_for(t->device);
     if (!scratch) return ZL_ERR_CUDA;
     return zl_coalesced_attn_bwd(t, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, ZL_NOALLOC_SCRATCH_BYTES, stream);
 }
@@ -603,6 +554,7 @@ zl_status zl_debug_set_fwd_order(zl_tasks* t, int32_t mode, void* stream) {
 zl_status zl_selftest_bounded_wait(const zl_tasks* t, int32_t limit_us, void* stream) {
     if (!t) return ZL_ERR_INVALID_ARG;
     if (t->device < 0) return ZL_ERR_CUDA;
+    if (!on_handle_device(t)) return ZL_ERR_INVALID_ARG;
     const int32_t us = limit_us < 1 ? 1 : (limit_us > 100000 ? 100000 : limit_us);
     if (launch_wait_selftest(t->d_status, (uint64_t)us * 1000ull, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return ZL_ERR_CUDA;

@@ -194,59 +194,20 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
     if (atomicCAS(status, 0, (int)ZL_ERR_TIMEOUT) == 0) status[1] = where;
 }
 
-#ifdef ZL_PROFILE
-// Development aid (profile builds only): cycles spent waiting at each site and in each MMA
-// issue segment, for the first CTAs.
-#ifdef ZL_TRACE_ONLY
-#define ZL_PROF_T0
-#define ZL_PROF_ADD(site)
-#define ZL_PROF_MARK(site)
-#else
-#define ZL_PROF_T0 const long long prof_t0_ = clock64();
-#define ZL_PROF_ADD(site) \
-    if (p.prof && blockIdx.x < 4 && lane == 0) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_t0_));
-#define ZL_PROF_MARK(site) \
-    if (p.prof && blockIdx.x < 4 && warp == 4 && lane == 0) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_seg_));
-#endif
-// Event trace: timestamp of event `ev` (0..15) of role `role` (0 MMA, 1 P/dS warp 4, 2 dQ warp 12) for
-// global iterations 200..207 of CTA 0.
-#define ZL_TRACE(role, ev, itc) \
-    if (p.prof && blockIdx.x == 0 && (itc) >= 200u && (itc) < 208u) p.prof[256 + (role) * 128 + ((itc) - 200u) * 16 + (ev)] = clock64();
-#ifdef ZL_TRACE_ONLY
-#define ZL_PROF_SEG_BEGIN
-#define ZL_PROF_SEG_END(site)
-#else
-#define ZL_PROF_SEG_BEGIN const long long prof_seg_ = clock64();
-#define ZL_PROF_SEG_END(site) \
-    if (p.prof && blockIdx.x < 4) atomicAdd((unsigned long long*)&p.prof[(blockIdx.x * 64 + (site))], (unsigned long long)(clock64() - prof_seg_));
-#endif
-#else
-#define ZL_PROF_T0
-#define ZL_PROF_ADD(site)
-#define ZL_PROF_SEG_BEGIN
-#define ZL_PROF_SEG_END(site)
-#define ZL_PROF_MARK(site)
-#define ZL_TRACE(role, ev, itc)
-#endif
-
 #define ZL_WAIT(bar, parity, site)                                        \
     do {                                                                  \
-        ZL_PROF_T0                                                        \
         if (!mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag)) { \
             report(p.status, &sm.abort_flag, 2000 + (site));              \
             goto teardown;                                                \
         }                                                                 \
-        ZL_PROF_ADD(site)                                                 \
     } while (0)
 #define ZL_WAIT_WARP(bar, parity, site)                                              \
     do {                                                                             \
-        ZL_PROF_T0                                                                   \
         const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag); \
         if (!__all_sync(0xffffffffu, ok_)) {                                         \
             report(p.status, &sm.abort_flag, 2000 + (site));                         \
             goto teardown;                                                           \
         }                                                                            \
-        if (warp == 4 || warp == 12) { ZL_PROF_ADD(site) }                           \
     } while (0)
 
 // Number of 128-row query tiles a kv group's CTA iterates over.
@@ -321,9 +282,6 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-#ifdef ZL_PROFILE
-    const long long prof_start = clock64();
-#endif
 
     if (warp < 4) {
         reg_dec<104>();
@@ -385,7 +343,6 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             constexpr uint32_t kQStageStep = Smem::kTileBytes >> 4, kAugStageStep = 4096 >> 4;
             // S^T = K Q^T - LSE/scale: the last step multiplies the ones block with the LSE pieces
             auto issue_s = [&](uint32_t stage) {
-                ZL_PROF_SEG_BEGIN
                 const uint64_t dq = dq_k0 + stage * kQStageStep;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
@@ -394,11 +351,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 if (mma_lane) mma_ss(tmem + kColS, dones_s, daug0 + stage * kAugStageStep, idesc_s, true);
                 if (mma_lane) mma_commit(&sm.s_full);
-                ZL_PROF_SEG_END(40)
             };
             // dP^T = V dO^T - D: the ones sit in the second K chunk, where the tile holds the D pieces
             auto issue_dp = [&](uint32_t stage) {
-                ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
@@ -406,16 +361,13 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 if (mma_lane) mma_ss(tmem + kColDP, dones_dp, daug0 + stage * kAugStageStep, idesc_s, true);
                 if (mma_lane) mma_commit(&sm.dp_full);
-                ZL_PROF_SEG_END(41)
             };
             auto issue_dv = [&](bool acc) {
-                ZL_PROF_SEG_BEGIN
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
                     if (mma_lane) mma_ts(tmem + kColDV, tmem + kColS + (ks / 4) * 64 + (ks % 4) * 8, ddo_mn + ks * (2048 >> 4), idesc_dv,
                            acc || ks > 0);
                 if (mma_lane) mma_commit(&sm.do_empty);
-                ZL_PROF_SEG_END(42)
             };
             uint32_t item_cnt = 0, it_cnt = 0;
             for (int it = blockIdx.x; it < p.n_items; it += gridDim.x, ++item_cnt) {
@@ -443,17 +395,13 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     const uint64_t dq_mn = dq_mn0 + (it_cnt & 1) * kQStageStep;
-                    ZL_TRACE(0, 0, it_cnt)
                     ZL_WAIT_WARP(&sm.ds_full, it_cnt & 1, 17);
-                    ZL_TRACE(0, 1, it_cnt)
                     tc_fence_after();
                     {
-                        ZL_PROF_SEG_BEGIN
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)  // dQ = dS K, K = 128 key rows; lands in the dP columns
                             if (mma_lane) mma_ss(tmem + kColDP, dds_mn + ks * (2048 >> 4), dk_mn + ks * (2048 >> 4), idesc_dq, ks > 0);
                         if (mma_lane) mma_commit(&sm.dq_full);  // dQ first: its drain from TMEM runs under the dK MMAs
-                        ZL_TRACE(0, 2, it_cnt)
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {  // dK += dS^T Q, K = 128 query rows
                             const uint32_t off = ((ks / 4) * Smem::kBoxBytes + (ks % 4) * 32) >> 4;
@@ -461,29 +409,20 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         }
                         if (mma_lane) mma_commit(&sm.q_empty[it_cnt & 1]);
                         if (mma_lane) mma_commit(&sm.ds_free);
-                        ZL_PROF_SEG_END(43)
                     }
-                    ZL_TRACE(0, 3, it_cnt)
                     if (i + 1 < n_it) {
                         const uint32_t n1 = it_cnt + 1, n2 = it_cnt + 2;
                         ZL_WAIT_WARP(&sm.do_full, n1 & 1, 18);
-                        ZL_TRACE(0, 4, it_cnt)
                         ZL_WAIT_WARP(&sm.dq_empty, it_cnt & 1, 19);
-                        ZL_TRACE(0, 5, it_cnt)
                         tc_fence_after();
                         issue_dp(n1 & 1);
-                        ZL_TRACE(0, 6, it_cnt)
                         ZL_WAIT_WARP(&sm.p_full, n1 & 1, 20);
-                        ZL_TRACE(0, 7, it_cnt)
                         tc_fence_after();
                         issue_dv(true);
-                        ZL_TRACE(0, 8, it_cnt)
                         if (i + 2 < n_it) {
                             ZL_WAIT_WARP(&sm.q_full[n2 & 1], (n2 >> 1) & 1, 16);
-                            ZL_TRACE(0, 9, it_cnt)
                             tc_fence_after();
                             issue_s(n2 & 1);
-                            ZL_TRACE(0, 10, it_cnt)
                         }
                     }
                 }
@@ -514,19 +453,14 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
                     const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
                     const bool tile_full = (wi.rows == kTileKV) && (q_valid == kTileQ);  // warp-uniform
-                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 0, it_cnt) }
                     ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 22);
-                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 1, it_cnt) }
                     tc_fence_after();
-                    ZL_PROF_SEG_BEGIN
                     uint32_t pk[32];  // P^T of this thread's row, bf16 pairs
                     {
                         uint32_t sr[2][32];
                         tmem_ld_x32(lane_addr + kColS + col0, sr[0]);
                         tmem_ld_x32(lane_addr + kColS + col0 + 32, sr[1]);
                         tmem_wait_ld();
-                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 6, it_cnt) }
-                        ZL_PROF_MARK(46)
                         if (tile_full) {
 #pragma unroll
                             for (int c = 0; c < 2; ++c)
@@ -548,18 +482,13 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                 }
                             }
                         }
-                        ZL_PROF_MARK(47)
                         tmem_st_x32(lane_addr + kColS + col0, pk);
-                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 7, it_cnt) }
                     }
                     tmem_wait_st();
-                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 8, it_cnt) }
                     tc_fence_before();
                     mbar_arrive(&sm.p_full);
-                    if (warp == 4 && lane == 0) { ZL_PROF_SEG_END(44) ZL_TRACE(1, 2, it_cnt) }
 
                     ZL_WAIT_WARP(&sm.dp_full, it_cnt & 1, 23);
-                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 3, it_cnt) }
                     if (it_cnt > 0) ZL_WAIT_WARP(&sm.ds_free, (it_cnt - 1) & 1, 24);  // dS buffer consumed by dK/dQ
                     if (store_pending) {
                         // this warpgroup's box of the dS tile staged the previous item's dK / dV tile
@@ -567,16 +496,12 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         named_bar_sync(2 + wg, 128);
                         store_pending = false;
                     }
-                    if (warp == 4 && lane == 0) { ZL_TRACE(1, 4, it_cnt) }
                     tc_fence_after();
                     {
-                        ZL_PROF_SEG_BEGIN
                         uint32_t dr[2][32];
                         tmem_ld_x32(lane_addr + kColDP + col0, dr[0]);
                         tmem_ld_x32(lane_addr + kColDP + col0 + 32, dr[1]);
                         tmem_wait_ld();
-                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 9, it_cnt) }
-                        ZL_PROF_MARK(48)
 #pragma unroll
                         for (int c = 0; c < 2; ++c) {
                             uint32_t dd[16];
@@ -602,12 +527,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                 st_shared_v4(addr, dd[k4 * 4], dd[k4 * 4 + 1], dd[k4 * 4 + 2], dd[k4 * 4 + 3]);
                             }
                         }
-                        ZL_PROF_MARK(49)
-                        if (warp == 4 && lane == 0) { ZL_TRACE(1, 10, it_cnt) }
                         tc_fence_before();
                         fence_proxy_async_smem();
                         mbar_arrive(&sm.ds_full);
-                        if (warp == 4 && lane == 0) { ZL_PROF_SEG_END(45) ZL_TRACE(1, 5, it_cnt) }
                     }
                 }
             }
@@ -689,9 +611,7 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                 const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
-                    if (warp == 12 && lane == 0) { ZL_TRACE(2, 0, it_cnt) }
                     ZL_WAIT_WARP(&sm.dq_full, it_cnt & 1, 31);
-                    if (warp == 12 && lane == 0) { ZL_TRACE(2, 1, it_cnt) }
                     tc_fence_after();
                     {
                         // read the whole tile (frees the TMEM columns for the next dP^T), then stage
@@ -707,7 +627,6 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         tmem_wait_ld();
                         tc_fence_before();
                         mbar_arrive(&sm.dq_empty);
-                        if (warp == 12 && lane == 0) { ZL_TRACE(2, 2, it_cnt) }
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c, ++chunk_cnt) {
                             // each warp stages its own 32 rows and adds them with its own reduce: no
@@ -737,9 +656,9 @@ zl_bwd_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
 
 teardown:
-#ifdef ZL_PROFILE
-    if (p.prof && blockIdx.x < 4 && threadIdx.x == 32) p.prof[blockIdx.x * 64 + 0] = clock64() - prof_start;
-#endif
+    // Also reached after an expired wait: bulk stores and reduces this thread has committed must have
+    // finished reading shared memory before the CTA gives it up (a no-op on the normal path).
+    bulk_wait_group<0>();
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -749,16 +668,22 @@ teardown:
     }
 }
 
+// The opt-in to large dynamic shared memory is a per-device attribute of the kernel.
+constexpr int kMaxDevices = 64;
+
 template <int D>
 cudaError_t launch_main_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                           const CUtensorMap& tdo, const CUtensorMap& tdq, const CUtensorMap& tdk,
                           const CUtensorMap& tdv, const BwdParams& p, int grid, cudaStream_t stream) {
     constexpr int smem = sizeof(BwdSmem<D>);
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(zl_bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    static bool configured[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+        e = cudaFuncSetAttribute(zl_bwd_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
     }
     zl_bwd_main_kernel<D><<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, tdq, tdk, tdv, p);
     return cudaGetLastError();

@@ -22,7 +22,6 @@ struct FwdParams {
     float* o_partial;
     float* lse_partial;
     int32_t* status;  // [0] = code, [1] = where
-    long long* prof;  // development aid (ZL_PROFILE builds), else null
 };
 
 struct MergeParams {
@@ -62,7 +61,6 @@ struct BwdParams {
     float* dq_acc;  // [q_pad_total, H, d]
     uint8_t* aug;   // [H, q_pad_total / 128] tiles of 4 KB: bf16 splits of -lse/scale and -rowsum(dO o O)
     int32_t* status;
-    long long* prof;  // development aid (ZL_PROFILE builds), else null
 };
 
 cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);

@@ -54,14 +54,6 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
     if (atomicCAS(status, 0, (int)ZL_ERR_TIMEOUT) == 0) status[1] = where;
 }
 
-#ifdef ZL_PROFILE
-// Development aid (profile builds only): timestamps of event `ev` of role `role` (0 MMA warp,
-// 1 / 2 softmax warp 4 / 8) for key-tile iterations 200..207 of CTA 0.
-#define ZL_TRACE(role, ev, itc) \
-    if (p.prof && blockIdx.x == 0 && lane == 0 && (itc) >= 200u && (itc) < 208u) p.prof[256 + (role) * 128 + ((itc) - 200u) * 16 + (ev)] = clock64();
-#else
-#define ZL_TRACE(role, ev, itc)
-#endif
 
 // Wait used by a single elected thread.
 #define ZL_WAIT(bar, parity, site)                                        \
@@ -225,39 +217,31 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     const bool has_next = j + 1 < n_kv;
                     // tile A: P_A(j) is in TMEM (S_A(j) fully read, O_A rescaled if needed); K(j), V(j)
                     // were waited for when S(j) was issued
-                    ZL_TRACE(0, 0, kv_cnt)
                     ZL_WAIT_WARP(&sm.p_half[0][0], pa_cnt & 1, 14);
                     tc_fence_after();
                     issue_pv(0, s, j > 0, 0);
                     ZL_WAIT_WARP(&sm.p_half[0][1], pa_cnt & 1, 15);
-                    ZL_TRACE(0, 1, kv_cnt)
                     ++pa_cnt;
                     tc_fence_after();
                     issue_pv(0, s, true, 1);
-                    ZL_TRACE(0, 2, kv_cnt)
                     if (!has_next) if (mma_lane) mma_commit(&sm.o_full[0]);
                     if (has_next) {
                         ZL_WAIT_WARP(&sm.kv_full[sn], (nk / kStages) & 1, 16);
-                        ZL_TRACE(0, 3, kv_cnt)
                         issue_s(0, sn);  // overwrites P_A(j): ordered after P_A V on the tensor pipe
-                        ZL_TRACE(0, 4, kv_cnt)
                     }
                     if (has_b) {
                         ZL_WAIT_WARP(&sm.p_half[1][0], pb_cnt & 1, 17);
                         tc_fence_after();
                         issue_pv(1, s, j > 0, 0);
                         ZL_WAIT_WARP(&sm.p_half[1][1], pb_cnt & 1, 18);
-                        ZL_TRACE(0, 5, kv_cnt)
                         ++pb_cnt;
                         tc_fence_after();
                         issue_pv(1, s, true, 1);
-                        ZL_TRACE(0, 6, kv_cnt)
                         if (!has_next) if (mma_lane) mma_commit(&sm.o_full[1]);
                     }
                     if (mma_lane) mma_commit(&sm.kv_empty[s]);  // S_A(j), S_B(j), P_A V(j), P_B V(j) are the stage's last readers
                     if (has_next) {
                         if (has_b) issue_s(1, sn);
-                        ZL_TRACE(0, 7, kv_cnt)
                         if (j + 2 == n_kv) if (mma_lane) mma_commit(&sm.q_empty);  // last S of the item issued
                     }
                 }
@@ -283,9 +267,7 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const int n_kv = (t.kv_len + kTileKV - 1) / kTileKV;
             float m_ref = -INFINITY, l = 0.f;  // reference maximum (raw score units) and row sum
             for (int j = 0; j < n_kv; ++j) {
-                if (quarter == 0) { ZL_TRACE(1 + x, 0, s_cnt) }
                 ZL_WAIT_WARP(&sm.s_full[x], s_cnt & 1, 21);
-                if (quarter == 0) { ZL_TRACE(1 + x, 1, s_cnt) }
                 ++s_cnt;
                 tc_fence_after();
                 float sv[kTileKV];
@@ -297,7 +279,6 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     for (int i = 0; i < 32; ++i) sv[c * 32 + i] = __uint_as_float(r[i]);
                 }
                 tmem_wait_ld();
-                if (quarter == 0) { ZL_TRACE(1 + x, 2, s_cnt - 1) }
                 const int valid = t.kv_len - j * kTileKV;  // columns of this tile inside the task
                 if (valid < kTileKV) {
 #pragma unroll
@@ -338,7 +319,6 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     if (j == 0) l = 0.f;
                     m_ref = mx;
                 }
-                if (quarter == 0) { ZL_TRACE(1 + x, 3, s_cnt - 1) }
                 const float nmb = -m_ref * sl2;
                 float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
@@ -356,10 +336,8 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(&sm.p_half[x][h]);
-                    if (quarter == 0) { ZL_TRACE(1 + x, 4 + h, s_cnt - 1) }
                 }
                 l += sum2.x + sum2.y;
-                if (quarter == 0) { ZL_TRACE(1 + x, 6, s_cnt - 1) }
             }
             // ---- epilogue
             const bool row_ok = row < tile_rows;
@@ -488,6 +466,9 @@ zl_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
 
 teardown:
+    // Also reached after an expired wait: bulk stores this thread has committed must have finished
+    // reading shared memory before the CTA gives it up (a no-op on the normal path).
+    bulk_wait_group<0>();
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -501,11 +482,16 @@ template <int D>
 cudaError_t launch_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                      const CUtensorMap& top, const FwdParams& p, int grid, cudaStream_t stream) {
     constexpr int smem = sizeof(FwdSmem<D>);
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(zl_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+    constexpr int kMaxDevices = 64;
+    static bool configured[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+        e = cudaFuncSetAttribute(zl_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
     }
     zl_fwd_kernel<D><<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, to, top, p);
     return cudaGetLastError();
