@@ -1,9 +1,19 @@
 """GPU parity on the five named configurations at full size, in the launch configuration the
-benchmark times.  Configurations 1-3 are compared on every head, row and column; 4 and 5
-on a set of full heads plus, for the other heads, stratified sample rows (O, LSE, dQ are
-row-local given all keys) and sum invariants that hold for any input
-(sum_j dV_j = sum_i dO_i and sum_j dK_j = 0 over each sequence's key set)."""
+benchmark times.
+
+Configurations 1-3 are compared on every head, row and column.  Configurations 4 and 5 are
+compared on a set of heads whose forward the oracle evaluates on every row (O and LSE everywhere),
+with dQ on stratified query rows and dK/dV on stratified key rows, element by element -- both are
+exact given the head's full LSE and D -- plus, for further heads, stratified sample rows of O, LSE
+and dQ and the sum identities that hold for any input (sum_j dV_j = sum_i dO_i, sum_j dK_j = 0).
+"Stratified" means: first and last row, both sides of every chunk boundary, both sides of the start
+of every ragged last 128-row tile, the whole ragged tail when it is short, and seeded random rows.
+
+Spike variants of configurations 3-5 plant keys aligned with chosen queries at the first and last
+key of every chunk and around the last tile of every chunk, so that a dropped, duplicated or
+leaked key is an O(1) error instead of one part in tens of thousands."""
 import os
+import time
 
 import numpy as np
 import pytest
@@ -11,20 +21,20 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as A
-from zl_testlib import (GpuRun, check_backward, check_forward, dev_to_f64, rel_fro, to_dev, to_f64,
-                        TOL_GRAD_REL, TOL_LSE_MAX, TOL_O_MAX, TOL_O_MEAN)
+from zl_testlib import (GpuRun, check_backward, check_forward, dev_to_f64, rel_fro, row_rel, to_dev, to_f64,
+                        TOL_GRAD_REL, TOL_GRAD_ROW, TOL_LSE_MAX, TOL_O_MAX, TOL_O_MEAN)
 
 pytestmark = pytest.mark.gpu
 WORKERS = min(16, len(os.sched_getaffinity(0)))
 
 
-def _inputs(p, heads=None):
+def _inputs(p, heads=None, tensors=("Q", "K", "V", "dO")):
     """Host bf16 bit patterns per tensor and head from the canonical generator: {tensor: {head: [rows, d]}}.
     With `heads` given, only those heads are generated on the host (the others are filled on the
     device with seeded normals that no check reads)."""
     hs = list(range(p.n_heads)) if heads is None else sorted(set(heads))
     import concurrent.futures as cf
-    out = {t: {} for t in ("Q", "K", "V", "dO")}
+    out = {t: {} for t in tensors}
     with cf.ProcessPoolExecutor(max_workers=WORKERS) as ex:
         futs = {(t, h): ex.submit(W._head_bits, p.seed, t, h, W.rows_of(p, t), p.head_dim) for t in out for h in hs}
         for (t, h), f in futs.items():
@@ -32,10 +42,11 @@ def _inputs(p, heads=None):
     return out
 
 
-def _run_gpu(p, B):
-    run = GpuRun(p)
+def _device_tensors(p, B):
     d = {}
     for i, t in enumerate(("Q", "K", "V", "dO")):
+        if t not in B:
+            continue
         rows = W.rows_of(p, t)
         if len(B[t]) == p.n_heads:
             x = torch.empty((rows, p.n_heads, p.head_dim), dtype=torch.bfloat16, device="cuda")
@@ -44,6 +55,12 @@ def _run_gpu(p, B):
         for h, bits_h in B[t].items():
             x[:, h, :] = to_dev(bits_h)
         d[t] = x
+    return d
+
+
+def _run_gpu(p, B):
+    run = GpuRun(p)
+    d = _device_tensors(p, B)
     O, LSE, _, _ = run.forward(d["Q"], d["K"], d["V"])
     dQ, dK, dV = run.backward(d["Q"], d["K"], d["V"], O, LSE, d["dO"])
     return O, LSE, dQ, dK, dV
@@ -53,9 +70,12 @@ def _head_src(B, t):
     return lambda h: W.bf16_bits_to_f32(B[t][h]).astype(np.float64)
 
 
-@pytest.mark.parametrize("ci", [1, 2])
+@pytest.mark.parametrize("ci", [1, 2, 3])
 def test_config_full_comparison(ci):
+    """Every head, every row, every column, forward and backward (graded tolerances plus the
+    row-wise gradient gate of check_backward)."""
     p = W.config(ci)
+    t0 = time.time()
     B = _inputs(p)
     O, LSE, dQ, dK, dV = _run_gpu(p, B)
     src = {t: _head_src(B, t) for t in B}
@@ -63,22 +83,36 @@ def test_config_full_comparison(ci):
     fs = check_forward(p, O, LSE, ref_f)
     ref_b = A.placement_bwd(p, src["Q"], src["K"], src["V"], src["dO"])
     bs = check_backward(p, dQ, dK, dV, ref_b)
-    print(f"config {ci}: all {p.n_heads} heads, every row: {fs} {bs}")
+    print(f"config {ci}: all {p.n_heads} heads, every row: {fs} {bs} ({time.time() - t0:.0f} s)")
 
 
-def _sample_rows(rng, n, k=48):
-    """First, last, rows around the ragged last tile, and seeded random rows."""
-    fixed = {0, n - 1, max(0, n - (n % 128 or 128)), max(0, n - (n % 128 or 128) - 1), min(n - 1, 127), min(n - 1, 128)}
-    extra = set(int(x) for x in rng.randint(0, n, size=max(0, k - len(fixed))))
-    return np.array(sorted(fixed | extra), dtype=np.int64)
+def _stratified(rng, n, chunk, k):
+    """Row indices of a range of n rows made of chunks of `chunk` rows (chunk = n: one chunk)."""
+    rows = {0, n - 1}
+    for c0 in range(0, n, chunk):
+        c1 = min(n, c0 + chunk)
+        tail0 = c0 + ((c1 - c0 - 1) // 128) * 128          # first row of the chunk's last 128-row tile
+        rows.update((c0, c1 - 1, tail0, min(c1 - 1, c0 + 127), min(c1 - 1, c0 + 128)))
+        if c0 > 0:
+            rows.add(c0 - 1)
+        if tail0 > c0:
+            rows.add(tail0 - 1)
+        if c1 - tail0 <= 32:
+            rows.update(range(tail0, c1))                   # a short ragged tail: every row of it
+    extra = max(0, k - len(rows))
+    rows.update(int(x) for x in rng.randint(0, n, size=extra))
+    return np.array(sorted(r for r in rows if 0 <= r < n), dtype=np.int64)
 
 
-def _check_sampled(ci, full_heads, fwd_full_heads, n_sample_heads, invariant_heads, host_heads=None):
+def _check_sampled(ci, full_heads, fwd_full_heads, n_sample_heads, invariant_heads, host_heads=None,
+                   n_long=256, n_short=24):
     """full_heads: forward and backward compared on every row / column.
-    fwd_full_heads: forward on every row; dQ on sampled rows and dK/dV on sampled key rows, which
-    are exact given the head's full LSE and D.  Other sampled heads: O, LSE, dQ on sampled rows.
-    invariant_heads: sum identities evaluated on the GPU's dK / dV."""
+    fwd_full_heads: forward on every row; dQ on stratified rows and dK/dV on stratified key rows, element
+    by element (exact given the head's full LSE and D).  Other sampled heads: O, LSE, dQ on stratified rows.
+    invariant_heads: sum identities evaluated on the GPU's dK / dV.
+    n_long / n_short: sample sizes per shard problem / per whole sequence."""
     p = W.config(ci)
+    t0 = time.time()
     rng = np.random.RandomState(100 + ci)
     others = [h for h in range(p.n_heads) if h not in full_heads and h not in fwd_full_heads]
     sample_heads = sorted(rng.choice(others, size=min(n_sample_heads, len(others)), replace=False).tolist())
@@ -101,26 +135,36 @@ def _check_sampled(ci, full_heads, fwd_full_heads, n_sample_heads, invariant_hea
         o_h = np.ascontiguousarray(ref_f["O"][:, 0, :]); lse_h = ref_f["LSE"][0]
         D_h = A.bwd_delta(do, o_h)
         dKg = dev_to_f64(dK[:, h, :]); dVg = dev_to_f64(dV[:, h, :]); dQg = dev_to_f64(dQ[:, h, :])
-        nk = dk_ = nv = dv_ = nq = dq_ = 0.0
+        got = {n: [] for n in ("dQ", "dK", "dV")}
+        want = {n: [] for n in ("dQ", "dK", "dV")}
+        n_rows = n_cols = 0
         for pr in probs:
             qo, ql = pr["q_off"], pr["q_len"]
             kk = np.concatenate([k[o:o + l] for o, l in pr["kv_ranges"]])
             vv = np.concatenate([v[o:o + l] for o, l in pr["kv_ranges"]])
             pos = np.concatenate([np.arange(o, o + l) for o, l in pr["kv_ranges"]])
-            cols = _sample_rows(rng, kk.shape[0], 96 if pr["shards"] else 16)
+            chunk = pr["kv_ranges"][0][1] if pr["shards"] else kk.shape[0]
+            cols = _stratified(rng, kk.shape[0], chunk, n_long if pr["shards"] else n_short)
             gk, gv = A.attn_bwd_dkdv(q[qo:qo + ql], kk, vv, do[qo:qo + ql], lse_h[qo:qo + ql], D_h[qo:qo + ql],
                                      p.scale, cols=cols)
-            nk += float(np.sum((dKg[pos[cols]] - gk) ** 2)); dk_ += float(np.sum(gk ** 2))
-            nv += float(np.sum((dVg[pos[cols]] - gv) ** 2)); dv_ += float(np.sum(gv ** 2))
-            rows = _sample_rows(rng, ql, 64 if pr["shards"] else 16)
+            got["dK"].append(dKg[pos[cols]]); want["dK"].append(gk)
+            got["dV"].append(dVg[pos[cols]]); want["dV"].append(gv)
+            rows = _stratified(rng, ql, ql, n_long if pr["shards"] else n_short)
             gq = A.attn_bwd_dq(q[qo:qo + ql], kk, vv, do[qo:qo + ql], lse_h[qo:qo + ql], D_h[qo:qo + ql], p.scale,
                                rows=rows)
-            nq += float(np.sum((dQg[qo + rows] - gq) ** 2)); dq_ += float(np.sum(gq ** 2))
-        rel = dict(dQ=np.sqrt(nq / dq_), dK=np.sqrt(nk / dk_), dV=np.sqrt(nv / dv_))
+            got["dQ"].append(dQg[qo + rows]); want["dQ"].append(gq)
+            n_rows += rows.size; n_cols += cols.size
+        rel, rowwise = {}, {}
+        for n in got:
+            g, w = np.concatenate(got[n]), np.concatenate(want[n])
+            rel[n] = rel_fro(g, w)
+            rowwise[n] = row_rel(g, w)
         assert max(rel.values()) <= TOL_GRAD_REL, rel
-        report.append(f"head {h}: forward on every row {fs}; sampled gradient rows/columns {rel}")
+        assert max(rowwise.values()) <= TOL_GRAD_ROW, rowwise
+        report.append(f"head {h}: forward on every row {fs}; dQ on {n_rows} rows, dK/dV on {n_cols} key rows "
+                      f"element by element: rel {rel} row-wise {rowwise}")
     # ---- other heads: sampled rows
-    eo, el, num, den = [], [], 0.0, 0.0
+    eo, el, gq_all, wq_all = [], [], [], []
     for h in sample_heads:
         q, k, v, do = (src[t](h) for t in ("Q", "K", "V", "dO"))
         Og = dev_to_f64(O[:, h, :]); Lg = dev_to_f64(LSE[h]); dQg = dev_to_f64(dQ[:, h, :])
@@ -128,20 +172,22 @@ def _check_sampled(ci, full_heads, fwd_full_heads, n_sample_heads, invariant_hea
             qo, ql = pr["q_off"], pr["q_len"]
             kk = np.concatenate([k[o:o + l] for o, l in pr["kv_ranges"]])
             vv = np.concatenate([v[o:o + l] for o, l in pr["kv_ranges"]])
-            rows = _sample_rows(rng, ql, 16 if not pr["shards"] else 64)
+            rows = _stratified(rng, ql, ql, 64 if pr["shards"] else 16)
             o_s, l_s = A.attn_fwd(q[qo:qo + ql], kk, vv, p.scale, rows=rows)
             eo.append(np.abs(Og[qo + rows] - o_s)); el.append(np.abs(Lg[qo + rows] - l_s))
             lse_full = np.zeros(ql); D_full = np.zeros(ql)
             lse_full[rows] = l_s
             D_full[rows] = np.sum(do[qo + rows] * o_s, axis=1)
             dq_s = A.attn_bwd_dq(q[qo:qo + ql], kk, vv, do[qo:qo + ql], lse_full, D_full, p.scale, rows=rows)
-            num += float(np.sum((dQg[qo + rows] - dq_s) ** 2)); den += float(np.sum(dq_s ** 2))
+            gq_all.append(dQg[qo + rows]); wq_all.append(dq_s)
     if sample_heads:
         eo = np.concatenate(eo); el = np.concatenate(el)
+        gq_all = np.concatenate(gq_all); wq_all = np.concatenate(wq_all)
         assert eo.max() <= TOL_O_MAX and eo.mean() <= TOL_O_MEAN and el.max() <= TOL_LSE_MAX
-        assert np.sqrt(num / den) <= TOL_GRAD_REL
+        assert rel_fro(gq_all, wq_all) <= TOL_GRAD_REL
+        assert row_rel(gq_all, wq_all) <= TOL_GRAD_ROW
         report.append(f"sampled heads {sample_heads}: O max {eo.max():.2e} mean {eo.mean():.2e} LSE max {el.max():.2e} "
-                      f"dQ rel {np.sqrt(num / den):.2e} on {eo.shape[0]} rows")
+                      f"dQ rel {rel_fro(gq_all, wq_all):.2e} row-wise {row_rel(gq_all, wq_all):.2e} on {eo.shape[0]} rows")
     # ---- sum invariants on the GPU's dK / dV.  sum_j dV_j = sum_i dO_i holds up to the bf16 rounding of
     # the stored elements; sum_j dK_j = scale * sum_i (dO_i . (O_i - O_i as stored in bf16)) q_i is zero only
     # up to the rounding of the stored O that D is computed from, hence the wider bound.
@@ -163,21 +209,81 @@ def _check_sampled(ci, full_heads, fwd_full_heads, n_sample_heads, invariant_hea
             assert ev <= tol_v, ("dV sum", h, pr["q_off"], ev, tol_v, rms_v, n_keys)
             assert np.abs(sk).max() <= tol_k, ("dK sum", h, pr["q_off"], np.abs(sk).max(), tol_k, rms_k, n_keys)
     report.append(f"dK/dV sum invariants on heads {list(invariant_heads)}")
-    print(f"config {ci}: " + "; ".join(report))
-
-
-def test_config3_full_heads_and_samples():
-    _check_sampled(3, full_heads=[0, 11], fwd_full_heads=[5], n_sample_heads=3, invariant_heads=range(12))
+    print(f"config {ci} ({time.time() - t0:.0f} s): " + "; ".join(report))
 
 
 def test_config4_full_heads_and_samples():
-    _check_sampled(4, full_heads=[0], fwd_full_heads=[39], n_sample_heads=4, invariant_heads=range(0, 40, 3))
+    _check_sampled(4, full_heads=[0], fwd_full_heads=[13, 26, 39], n_sample_heads=4, invariant_heads=range(0, 40, 3))
 
 
 @pytest.mark.slow
-def test_config5_full_head_and_samples():
-    # one full head of this configuration costs the plain oracle minutes (1.6e10 score pairs), so the
-    # long-video shard is checked on sampled rows of five heads plus the sum invariants; the kernels'
-    # dK/dV paths are compared column by column in configurations 1-4
-    _check_sampled(5, full_heads=[], fwd_full_heads=[], n_sample_heads=5, invariant_heads=[0, 39],
-                   host_heads="needed")
+def test_config5_full_forward_head_and_samples():
+    # head 0: the oracle evaluates the forward of the 31,110 x 497,760 problem on every row (minutes on the
+    # host cores), which makes dQ rows and dK/dV key rows exact one by one; the key rows sampled include both
+    # sides of all fifteen chunk boundaries and every row of each chunk's 6-row tail tile
+    _check_sampled(5, full_heads=[], fwd_full_heads=[0], n_sample_heads=4, invariant_heads=[0, 39],
+                   host_heads="needed", n_long=384)
+
+
+# --------------------------------------------------------------------------------------------------
+# Spike variants (forward): keys aligned with chosen queries at chunk and tile boundaries
+# --------------------------------------------------------------------------------------------------
+
+SPIKE_BETA = 8.0   # k_j = beta * q_i (exact in bf16): s_ij = beta * scale * |q_i|^2 ~ 90 at d = 128
+
+
+def _boundary_keys(off, length):
+    """First and last key of a K/V range and both sides of the start of its last 128-row tile."""
+    tail0 = off + ((length - 1) // 128) * 128
+    keys = [off, off + length - 1, tail0]
+    if tail0 > off:
+        keys.append(tail0 - 1)
+    return sorted(set(keys))
+
+
+@pytest.mark.parametrize("ci", [3, 4, 5])
+def test_spike_keys_at_chunk_and_tile_boundaries_full_size(ci):
+    p = W.config(ci)
+    t0 = time.time()
+    heads = [0, p.n_heads - 1]
+    B = _inputs(p, heads, tensors=("Q", "K", "V"))
+    rng = np.random.RandomState(500 + ci)
+    probs = A.logical_problems(p)
+    planted = {h: [] for h in heads}          # (query row, key row) in absolute coordinates
+    for h in heads:
+        qf = W.bf16_bits_to_f32(B["Q"][h])
+        kf = W.bf16_bits_to_f32(B["K"][h]).copy()
+        for pr in probs:
+            keys = [j for (o, l) in pr["kv_ranges"] for j in _boundary_keys(o, l)]
+            rows = pr["q_off"] + rng.choice(pr["q_len"], size=len(keys), replace=False)
+            for i, j in zip(rows.tolist(), keys):
+                kf[j] = SPIKE_BETA * qf[i]
+                planted[h].append((i, j))
+        B["K"][h] = W.f32_to_bf16_bits(kf)
+    d = _device_tensors(p, B)
+    run = GpuRun(p)
+    O, LSE, _, _ = run.forward(d["Q"], d["K"], d["V"])
+    n_checked = n_sharp = 0
+    worst_o = worst_l = 0.0
+    for h in heads:
+        q, k, v = (W.bf16_bits_to_f32(B[t][h]).astype(np.float64) for t in ("Q", "K", "V"))
+        Og = dev_to_f64(O[:, h, :]); Lg = dev_to_f64(LSE[h])
+        by_row = dict(planted[h])
+        for pr in probs:
+            qo, ql = pr["q_off"], pr["q_len"]
+            rows = np.array(sorted(i - qo for i in by_row if qo <= i < qo + ql), dtype=np.int64)
+            kk = np.concatenate([k[o:o + l] for o, l in pr["kv_ranges"]])
+            vv = np.concatenate([v[o:o + l] for o, l in pr["kv_ranges"]])
+            o_s, l_s = A.attn_fwd(q[qo:qo + ql], kk, vv, p.scale, rows=rows)
+            eo = np.abs(Og[qo + rows] - o_s); el = np.abs(Lg[qo + rows] - l_s)
+            assert eo.max() <= TOL_O_MAX and el.max() <= TOL_LSE_MAX, (ci, h, qo, float(eo.max()), float(el.max()))
+            worst_o = max(worst_o, float(eo.max())); worst_l = max(worst_l, float(el.max()))
+            for r, o_row in zip(rows.tolist(), o_s):
+                j = by_row[qo + r]
+                if np.abs(o_row - v[j]).max() < 1e-6:        # the oracle confirms the spike owns this row
+                    n_sharp += 1
+                    assert np.abs(Og[qo + r] - v[j]).max() <= TOL_O_MAX, (ci, h, qo + r, j)
+                n_checked += 1
+    assert n_sharp >= 0.9 * n_checked, (n_sharp, n_checked)
+    print(f"config {ci} spikes ({time.time() - t0:.0f} s): {n_checked} planted (query, key) pairs on heads {heads}, "
+          f"{n_sharp} with O_i = v_j in the oracle; O max err {worst_o:.2e}, LSE max err {worst_l:.2e}")

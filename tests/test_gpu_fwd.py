@@ -62,22 +62,26 @@ def test_tile_edge_lengths_shards(lq, lkv):
 
 def test_spike_keys_at_tile_and_chunk_boundaries():
     """A key aligned with a query makes that query's output equal that key's value row, so
-    a dropped, duplicated or leaked key is an O(1) error."""
+    a dropped, duplicated or leaked key is an O(1) error.  Keys of the NEIGHBOURING sequences (the
+    previous one's last key, the next one's first key) aligned with queries of this sequence must
+    have no effect at all."""
     d, H = 128, 1
-    p = W.make_placement("spike", H, d, 3, [300, 200], [(1, 2, 260)])
+    p = W.make_placement("spike", H, d, 3, [300, 200, 150], [(1, 2, 260)])
     rng = np.random.RandomState(9)
     Q = rng.standard_normal((p.total_q, H, d)).astype(np.float32)
     K = rng.standard_normal((p.total_kv, H, d)).astype(np.float32) * 0.1
     V = rng.standard_normal((p.total_kv, H, d)).astype(np.float32)
     beta = 4.0
     # (query row, key row) pairs inside the same logical problem
-    pairs = [(0, 0), (5, 127), (6, 128), (7, 255), (8, 256), (9, 299),          # whole seq 0 (300)
-             (300, 300), (301, 499),                                             # whole seq 1 (200)
-             (500, 500), (501, 627), (502, 628), (503, 759), (504, 760), (505, 1019)]  # shard chunks
-    for qi, kj in pairs:
+    pairs = [(0, 0), (5, 127), (6, 128), (7, 255), (8, 256), (9, 298),           # whole seq 0 (rows 0-299)
+             (300, 300), (301, 498),                                              # whole seq 1 (rows 300-499)
+             (505, 501), (506, 649),                                              # whole seq 2 (rows 500-649)
+             (650, 650), (651, 777), (652, 778), (653, 909), (654, 910), (655, 1169)]  # shard chunks
+    # (query row, key row of a NEIGHBOUR): seq 0's last key and seq 2's first key aligned with queries of
+    # seq 1, seq 1's last key aligned with a query of seq 2
+    foreign = [(310, 299), (311, 500), (510, 499)]
+    for qi, kj in pairs + foreign:
         K[kj] = beta * Q[qi]
-    # spikes in NEIGHBOURING problems must have no effect
-    K[300 - 1] = K[300 - 1]  # (last key of seq 0 is already a spike target of row 9)
     Qb, Kb, Vb = (W.f32_to_bf16_bits(W._bf16_round_f32(x)) for x in (Q, K, V))
     run, (O, LSE, OP, LP), ref, stats = _run(p, Qb, Kb, Vb, gate=False)
     Og = dev_to_f64(O)
@@ -85,6 +89,11 @@ def test_spike_keys_at_tile_and_chunk_boundaries():
     for qi, kj in pairs:
         assert np.abs(ref["O"][qi, 0] - Vf[kj, 0]).max() < 1e-6, "spike too weak for the test"
         assert np.abs(Og[qi, 0] - Vf[kj, 0]).max() < 2e-2, (qi, kj)
+    for qi, kj in foreign:
+        # had the foreign key leaked into the row's softmax, the row would equal its value row
+        assert np.abs(ref["O"][qi, 0] - Vf[kj, 0]).max() > 0.5
+        assert np.abs(Og[qi, 0] - ref["O"][qi, 0]).max() < 2e-2, (qi, kj)
+        assert np.abs(Og[qi, 0] - Vf[kj, 0]).max() > 0.5, (qi, kj)
 
 
 def test_isolation_and_untouched_rows():

@@ -13,6 +13,14 @@ TOL_O_MAX, TOL_O_MEAN, TOL_LSE_MAX, TOL_GRAD_REL = 2e-2, 2e-3, 1e-3, 1e-2
 # GATE_O_MAX bounds the error in excess of the output's own bf16 rounding (2^-8 * |O|).
 GATE_O_MAX, GATE_LSE_MAX, GATE_GRAD_REL = 3e-3, 2e-5, 5e-3
 
+# Row-wise gradient gate: a relative Frobenius norm over a whole tensor cannot see one wrong row among
+# tens of thousands, so every (row, head) vector g is also held to
+#     ||g - ref|| <= TOL_GRAD_ROW * (||ref|| + GRAD_ROW_FLOOR * rms),   rms = root mean square row norm of ref,
+# where the floor keeps rows whose own gradient is small relative to the tensor (their error is set by
+# the bf16 rounding of P and dS, which scales with the tensor, not with the row) from dividing by ~0.
+# GRAD_ROW_ABS covers tensors that are exactly zero in the oracle (a single key: dQ = dK = 0).
+TOL_GRAD_ROW, GRAD_ROW_FLOOR, GRAD_ROW_ABS = 3e-2, 0.1, 1e-3
+
 SENTINEL = 768.0  # exactly representable in bf16
 
 
@@ -123,7 +131,18 @@ def rel_fro(a, b):
     return float(np.linalg.norm(a - b) / nb) if nb > 0 else float(np.linalg.norm(a))
 
 
-def check_backward(p, dQ, dK, dV, ref, tol=TOL_GRAD_REL, heads=None):
+def row_rel(g, ref, rms=None):
+    """Largest row-wise relative error of g [..., d] against ref, with the floor described above.
+    `rms` (root mean square row norm of the whole tensor) may be given when ref is only a sample."""
+    rn = np.linalg.norm(ref, axis=-1)
+    if rn.size == 0:
+        return 0.0
+    if rms is None:
+        rms = float(np.sqrt(np.mean(rn ** 2)))
+    return float(np.max(np.linalg.norm(g - ref, axis=-1) / (rn + GRAD_ROW_FLOOR * rms + GRAD_ROW_ABS)))
+
+
+def check_backward(p, dQ, dK, dV, ref, tol=TOL_GRAD_REL, heads=None, row_tol=TOL_GRAD_ROW):
     hs = list(range(p.n_heads)) if heads is None else list(heads)
     qmask, kvmask = covered_rows(p)
     out = {}
@@ -131,6 +150,8 @@ def check_backward(p, dQ, dK, dV, ref, tol=TOL_GRAD_REL, heads=None):
         gg = dev_to_f64(g)[:, hs, :]
         out[name] = rel_fro(gg[mask], ref[name][mask])
         assert out[name] <= tol, (name, out)
+        out[name + "_row"] = row_rel(gg[mask], ref[name][mask])
+        assert out[name + "_row"] <= row_tol, (name, "row-wise", out)
         if (~mask).any():
             assert np.all(gg[~mask] == SENTINEL), f"{name}: rows outside every task were written"
     return out
