@@ -16,10 +16,12 @@ GATE_O_MAX, GATE_LSE_MAX, GATE_GRAD_REL = 3e-3, 2e-5, 5e-3
 # Row-wise gradient gate: a relative Frobenius norm over a whole tensor cannot see one wrong row among
 # tens of thousands, so every (row, head) vector g is also held to
 #     ||g - ref|| <= TOL_GRAD_ROW * (||ref|| + GRAD_ROW_FLOOR * rms),   rms = root mean square row norm of ref,
-# where the floor keeps rows whose own gradient is small relative to the tensor (their error is set by
-# the bf16 rounding of P and dS, which scales with the tensor, not with the row) from dividing by ~0.
+# where the floor keeps rows whose own gradient is small relative to the tensor from dividing by ~0: a
+# query whose softmax is nearly one-hot has a tiny dQ, yet its error is set by D = rowsum(dO o O) being
+# formed from the stored bf16 O (|dO . (O_bf16 - O)| ~ 1e-2 at d = 128), which does not shrink with the
+# row.  Measured: 0.04 * rms on such a row of a 2-token sequence, <= 0.01 elsewhere; a wrong row gives ~0.8.
 # GRAD_ROW_ABS covers tensors that are exactly zero in the oracle (a single key: dQ = dK = 0).
-TOL_GRAD_ROW, GRAD_ROW_FLOOR, GRAD_ROW_ABS = 3e-2, 0.1, 1e-3
+TOL_GRAD_ROW, GRAD_ROW_FLOOR, GRAD_ROW_ABS = 3e-2, 0.25, 1e-3
 
 SENTINEL = 768.0  # exactly representable in bf16
 
