@@ -123,6 +123,36 @@ zl_status zl_build_tasks_ex(const int32_t* cu_seqlens, int32_t n_whole,
                             int32_t total_q, int32_t total_kv, int32_t n_heads, int32_t head_dim,
                             uint32_t flags, void* stream, zl_tasks** out);
 
+/* zl_build_tasks_heads -- zl_build_tasks_ex for placements whose tasks cover different HEAD RANGES
+ * (Section IV-D, second coalescing mode: sequences under Ulysses parallelism hold all their tokens
+ * for n_heads / h of the heads, are batched with one QKV-packed all-to-all and run as one
+ * block-diagonal attention call; Table II, configuration (1, h, 1)).  Such tasks share one launch
+ * and one set of [tokens, n_heads, head_dim] buffers with tasks over all heads.
+ *
+ *   whole        host, n_whole descriptors: a sequence owning rows [off, off+len) of both token
+ *                spaces for heads [head_begin, head_begin+head_count).  Final after the forward
+ *                launch.  Unlike cu_seqlens, two whole sequences may own the same rows when their
+ *                head ranges are disjoint (two Ulysses sequences packed side by side in the head
+ *                dimension).  len = 0 is ignored.
+ *   shards       as in zl_build_tasks; shard_heads (host, n_shards entries, or NULL = all heads)
+ *                gives each shard's head range.  Shards lie at or after the end of the last whole
+ *                sequence.
+ * Validation, head by head: among the tasks that cover a head, query ranges are pairwise identical
+ * or disjoint and so are key ranges; tasks with an identical query range, or an identical key
+ * range, must have the same head range (ZL_ERR_OVERLAP otherwise).  Head ranges must satisfy
+ * 0 <= head_begin, 1 <= head_count, head_begin + head_count <= n_heads (ZL_ERR_INVALID_ARG).
+ * Merge groups, kv groups and the dQ accumulation units are formed per (range, head range); work
+ * items exist only for the heads of their task, and every (row, head) of every output that no
+ * task covers is left untouched.  Scratch and partial slots are sized for n_heads heads per row
+ * whatever the task's head count.
+ * zl_build_tasks_ex(cu_seqlens, ...) equals this call with whole[i] = (cu[i], cu[i+1]-cu[i], 0, n_heads). */
+typedef struct { int32_t off, len, head_begin, head_count; } zl_whole_desc;
+typedef struct { int32_t head_begin, head_count; } zl_head_range;
+zl_status zl_build_tasks_heads(const zl_whole_desc* whole, int32_t n_whole,
+                               const zl_shard_desc* shards, const zl_head_range* shard_heads, int32_t n_shards,
+                               int32_t total_q, int32_t total_kv, int32_t n_heads, int32_t head_dim,
+                               uint32_t flags, void* stream, zl_tasks** out);
+
 zl_status zl_tasks_get_info(const zl_tasks* tasks, zl_tasks_info* info);
 
 /* Slot of shard `shard_idx` (index into the `shards` array given to zl_build_tasks) inside
@@ -131,7 +161,9 @@ zl_status zl_tasks_get_info(const zl_tasks* tasks, zl_tasks_info* info);
 zl_status zl_tasks_get_partial_slot(const zl_tasks* tasks, int32_t shard_idx,
                                     int64_t* row_off, int64_t* rows_padded);
 
-/* Host copies of the work lists, for inspection and tests.  Each forward item is 4 int32:
+/* Host copies of the work lists, for inspection and tests.  Tasks are numbered in the order: whole
+ * sequences with len > 0, then shards with q_len > 0 (the shards of a fused range share one task).
+ * Each forward item is 4 int32:
  * (task, head, first query row of the block relative to the task, rows in the block); each
  * backward item is 4 int32: (kv group, head, first key row relative to the group, rows).
  * `items` may be NULL to query the count only. */

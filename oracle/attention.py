@@ -191,22 +191,37 @@ def _head(x: HeadSource, h: int) -> np.ndarray:
 def logical_problems(p) -> List[dict]:
     """Direct-form problems of a placement, in placement order.
 
-    Each entry: q_off, q_len, kv_ranges [(off, len), ...] in ascending shard order, and
-    ``shards`` (indices into p.shards; empty for a whole sequence)."""
+    Each entry: q_off, q_len, kv_ranges [(off, len), ...] in ascending shard order, ``shards``
+    (indices into p.shards; empty for a whole sequence) and ``heads`` = (head_begin, head_count): the
+    heads for which the problem exists (all heads unless the placement gives head ranges -- a
+    sequence under Ulysses parallelism holds its tokens for a subset of the heads; the attention of
+    each of those heads is the same definition)."""
     probs = []
-    for i in range(len(p.cu_seqlens) - 1):
-        a, b = p.cu_seqlens[i], p.cu_seqlens[i + 1]
-        probs.append(dict(q_off=a, q_len=b - a, kv_ranges=[(a, b - a)], shards=[]))
-    groups: Dict[Tuple[int, int], dict] = {}
+    if hasattr(p, "whole_descs"):
+        whole = p.whole_descs()
+        shard_heads = p.shard_head_ranges()
+    else:
+        whole = [(p.cu_seqlens[i], p.cu_seqlens[i + 1] - p.cu_seqlens[i], 0, p.n_heads)
+                 for i in range(len(p.cu_seqlens) - 1)]
+        shard_heads = [(0, p.n_heads)] * len(p.shards)
+    for (a, l, hb, hc) in whole:
+        probs.append(dict(q_off=a, q_len=l, kv_ranges=[(a, l)], shards=[], heads=(hb, hc)))
+    groups: Dict[Tuple[int, int, int, int], dict] = {}
     for si, (qo, ql, ko, kl, sid) in enumerate(p.shards):
-        g = groups.get((qo, ql))
+        hb, hc = shard_heads[si]
+        g = groups.get((qo, ql, hb, hc))
         if g is None:
-            g = dict(q_off=qo, q_len=ql, kv_ranges=[], shards=[])
-            groups[(qo, ql)] = g
+            g = dict(q_off=qo, q_len=ql, kv_ranges=[], shards=[], heads=(hb, hc))
+            groups[(qo, ql, hb, hc)] = g
             probs.append(g)
         g["kv_ranges"].append((ko, kl))
         g["shards"].append(si)
     return probs
+
+
+def _has_head(pr: dict, h: int) -> bool:
+    hb, hc = pr["heads"]
+    return hb <= h < hb + hc
 
 
 def _gather_kv(x: np.ndarray, ranges) -> np.ndarray:
@@ -237,6 +252,8 @@ def placement_fwd(p, Q: HeadSource, K: HeadSource, V: HeadSource, scale: Optiona
     for hi, h in enumerate(hs):
         q, k, v = _head(Q, h), _head(K, h), _head(V, h)
         for pr in probs:
+            if not _has_head(pr, h):
+                continue
             qo, ql = pr["q_off"], pr["q_len"]
             kk = _gather_kv(k, pr["kv_ranges"])
             vv = _gather_kv(v, pr["kv_ranges"])
@@ -277,6 +294,8 @@ def placement_bwd(p, Q: HeadSource, K: HeadSource, V: HeadSource, dO: HeadSource
     for hi, h in enumerate(hs):
         q, k, v, do = _head(Q, h), _head(K, h), _head(V, h), _head(dO, h)
         for pr in probs:
+            if not _has_head(pr, h):
+                continue
             qo, ql = pr["q_off"], pr["q_len"]
             kk = _gather_kv(k, pr["kv_ranges"])
             vv = _gather_kv(v, pr["kv_ranges"])
@@ -298,16 +317,19 @@ def placement_bwd_shard_form(p, Q, K, V, dO, scale=None, heads=None):
     d = p.head_dim
     fwd = placement_fwd(p, Q, K, V, scale, heads=hs, with_partials=False)
     dQ = np.zeros((p.total_q, len(hs), d)); dK = np.zeros((p.total_kv, len(hs), d)); dV = np.zeros_like(dK)
-    tasks = [(p.cu_seqlens[i], p.cu_seqlens[i + 1] - p.cu_seqlens[i],
-              p.cu_seqlens[i], p.cu_seqlens[i + 1] - p.cu_seqlens[i])
-             for i in range(len(p.cu_seqlens) - 1)] + [s[:4] for s in p.shards]
+    tasks = []
+    for pr in logical_problems(p):
+        if pr["shards"]:
+            tasks += [tuple(p.shards[si][:4]) + (pr["heads"],) for si in pr["shards"]]
+        else:
+            tasks.append((pr["q_off"], pr["q_len"], pr["q_off"], pr["q_len"], pr["heads"]))
     for hi, h in enumerate(hs):
         q, k, v, do = _head(Q, h), _head(K, h), _head(V, h), _head(dO, h)
         o_h = np.ascontiguousarray(fwd["O"][:, hi, :])
         D = bwd_delta(do, o_h)
         lse = np.ascontiguousarray(fwd["LSE"][hi])
-        for (qo, ql, ko, kl) in tasks:
-            if ql == 0 or kl == 0:
+        for (qo, ql, ko, kl, (hb, hc)) in tasks:
+            if ql == 0 or kl == 0 or not (hb <= h < hb + hc):
                 continue
             qs, ks, vs, dos = q[qo:qo + ql], k[ko:ko + kl], v[ko:ko + kl], do[qo:qo + ql]
             ls, Ds = lse[qo:qo + ql], D[qo:qo + ql]

@@ -32,6 +32,15 @@ class ShardDesc(ctypes.Structure):
                 ("kv_len", ctypes.c_int32), ("seq_id", ctypes.c_int32)]
 
 
+class WholeDesc(ctypes.Structure):
+    _fields_ = [("off", ctypes.c_int32), ("len", ctypes.c_int32), ("head_begin", ctypes.c_int32),
+                ("head_count", ctypes.c_int32)]
+
+
+class HeadRange(ctypes.Structure):
+    _fields_ = [("head_begin", ctypes.c_int32), ("head_count", ctypes.c_int32)]
+
+
 class TasksInfo(ctypes.Structure):
     _fields_ = [("n_tasks", ctypes.c_int32), ("n_merge_groups", ctypes.c_int32),
                 ("n_kv_groups", ctypes.c_int32), ("n_fwd_items", ctypes.c_int32),
@@ -55,6 +64,8 @@ def _load():
     lib.zl_build_tasks.argtypes = [vp, i32, vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
     lib.zl_build_tasks_ex.restype = ctypes.c_int
     lib.zl_build_tasks_ex.argtypes = [vp, i32, vp, i32, i32, i32, i32, i32, ctypes.c_uint32, vp, ctypes.POINTER(vp)]
+    lib.zl_build_tasks_heads.restype = ctypes.c_int
+    lib.zl_build_tasks_heads.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, ctypes.c_uint32, vp, ctypes.POINTER(vp)]
     lib.zl_tasks_get_info.restype = ctypes.c_int
     lib.zl_tasks_get_info.argtypes = [vp, ctypes.POINTER(TasksInfo)]
     lib.zl_tasks_get_partial_slot.restype = ctypes.c_int
@@ -212,6 +223,28 @@ def build_tasks(cu_seqlens: Sequence[int], shards: Sequence[Sequence[int]], tota
         st = _lib.zl_build_tasks(cu_p, n_whole, sh_p, len(shards), total_q, total_kv, n_heads, head_dim,
                                  _stream_ptr(stream), ctypes.byref(out))
     _check(st, "zl_build_tasks")
+    return TaskHandle(out.value, n_heads, head_dim, total_q, total_kv, len(shards))
+
+
+def build_tasks_heads(whole: Sequence[Sequence[int]], shards: Sequence[Sequence[int]],
+                      shard_heads: Optional[Sequence[Sequence[int]]], total_q: int, total_kv: int,
+                      n_heads: int, head_dim: int, stream=None, flags: int = 0) -> TaskHandle:
+    """zl_build_tasks_heads: whole = (off, len, head_begin, head_count) per whole sequence, shards =
+    (q_off, q_len, kv_off, kv_len, seq_id) per shard, shard_heads = (head_begin, head_count) per shard or
+    None for all heads."""
+    wd = (WholeDesc * max(1, len(whole)))(*[WholeDesc(*[int(v) for v in w]) for w in whole])
+    sh = (ShardDesc * max(1, len(shards)))(*[ShardDesc(*[int(v) for v in s[:5]]) for s in shards])
+    hr = None
+    if shard_heads is not None:
+        assert len(shard_heads) == len(shards)
+        hr = (HeadRange * max(1, len(shards)))(*[HeadRange(int(a), int(b)) for a, b in shard_heads])
+    out = ctypes.c_void_p()
+    st = _lib.zl_build_tasks_heads(ctypes.cast(wd, ctypes.c_void_p) if len(whole) else None, len(whole),
+                                   ctypes.cast(sh, ctypes.c_void_p) if len(shards) else None,
+                                   ctypes.cast(hr, ctypes.c_void_p) if hr is not None and len(shards) else None,
+                                   len(shards), total_q, total_kv, n_heads, head_dim, ctypes.c_uint32(flags),
+                                   _stream_ptr(stream), ctypes.byref(out))
+    _check(st, "zl_build_tasks_heads")
     return TaskHandle(out.value, n_heads, head_dim, total_q, total_kv, len(shards))
 
 

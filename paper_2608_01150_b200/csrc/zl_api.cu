@@ -160,11 +160,42 @@ zl_status zl_build_tasks_ex(const int32_t* cu_seqlens, int32_t n_whole, const zl
                             int32_t head_dim, uint32_t flags, void* stream, zl_tasks** out) {
     if (!out) return ZL_ERR_INVALID_ARG;
     *out = nullptr;
+    if (n_whole < 0 || (n_whole > 0 && !cu_seqlens)) return ZL_ERR_INVALID_ARG;
+    std::vector<zl_whole_desc> whole;
+    if (n_whole > 0) {
+        if (cu_seqlens[0] != 0) return ZL_ERR_INVALID_ARG;
+        for (int i = 0; i < n_whole; ++i) {
+            if (cu_seqlens[i + 1] < cu_seqlens[i]) return ZL_ERR_INVALID_ARG;
+            whole.push_back({cu_seqlens[i], cu_seqlens[i + 1] - cu_seqlens[i], 0, n_heads});
+        }
+    }
+    return zl_build_tasks_heads(whole.data(), n_whole, shards, nullptr, n_shards, total_q, total_kv, n_heads,
+                                head_dim, flags, stream, out);
+}
+
+zl_status zl_build_tasks_heads(const zl_whole_desc* whole, int32_t n_whole, const zl_shard_desc* shards,
+                               const zl_head_range* shard_heads, int32_t n_shards, int32_t total_q,
+                               int32_t total_kv, int32_t n_heads, int32_t head_dim, uint32_t flags,
+                               void* stream, zl_tasks** out) {
+    if (!out) return ZL_ERR_INVALID_ARG;
+    *out = nullptr;
     if (flags & ~ZL_BUILD_FUSE_LOCAL_CHUNKS) return ZL_ERR_INVALID_ARG;
+    if (n_whole < 0 || n_shards < 0 || (n_whole > 0 && !whole) || (n_shards > 0 && !shards)) return ZL_ERR_INVALID_ARG;
+    std::vector<InputTask> in;
+    in.reserve((size_t)n_whole + n_shards);
+    for (int i = 0; i < n_whole; ++i) {
+        const zl_whole_desc& w = whole[i];
+        if (w.off < 0 || w.len < 0 || (int64_t)w.off + w.len > std::min(total_q, total_kv)) return ZL_ERR_INVALID_ARG;
+        in.push_back({w.off, w.len, w.off, w.len, 0, w.head_begin, w.head_count, -1});
+    }
+    for (int i = 0; i < n_shards; ++i) {
+        const zl_shard_desc& d = shards[i];
+        const zl_head_range hr = shard_heads ? shard_heads[i] : zl_head_range{0, n_heads};
+        in.push_back({d.q_off, d.q_len, d.kv_off, d.kv_len, d.seq_id, hr.head_begin, hr.head_count, i});
+    }
     zl_tasks* h = new (std::nothrow) zl_tasks();
     if (!h) return ZL_ERR_INVALID_ARG;
-    zl_status st = build_schedule(cu_seqlens, n_whole, shards, n_shards, total_q, total_kv, n_heads, head_dim,
-                                  flags, &h->sched);
+    zl_status st = build_schedule(in, n_shards, total_q, total_kv, n_heads, head_dim, flags, &h->sched);
     if (st != ZL_OK) { delete h; return st; }
 
     int n_dev = 0;

@@ -73,6 +73,7 @@ __global__ void __launch_bounds__(kPreThreads) zl_bwd_pre_kernel(const BwdParams
         const int slot_row = row8 * 8 + sub;
         // slots are padded to 128 rows: the eight rows belong to one query group
         const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, row8 * 8)];
+        if (h < g.head_begin || h >= g.head_begin + g.head_count) continue;  // warp-uniform: no task runs this head
         const int r = slot_row - g.slot;
         float xd = 0.f, xl = -1e30f;
         const bool live = r < g.q_len;
@@ -134,15 +135,16 @@ __global__ void __launch_bounds__(kPreThreads) zl_bwd_post_kernel(const BwdParam
         if (r >= g.q_len) continue;
         const float* src = p.dq_acc + slot_row * p.n_heads * D + lane * V;
         __nv_bfloat16* dst = p.dq + ((int64_t)g.q_off + r) * p.grad_row_stride + lane * V;
-        for (int h0 = 0; h0 < p.n_heads; h0 += kBatch) {
+        const int h_end = g.head_begin + g.head_count;  // heads outside the group's range are left untouched
+        for (int h0 = g.head_begin; h0 < h_end; h0 += kBatch) {
             if constexpr (V == 4) {
                 float4 x[kBatch];
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i)
-                    if (h0 + i < p.n_heads) x[i] = __ldcs(reinterpret_cast<const float4*>(src + (int64_t)(h0 + i) * D));
+                    if (h0 + i < h_end) x[i] = __ldcs(reinterpret_cast<const float4*>(src + (int64_t)(h0 + i) * D));
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i)
-                    if (h0 + i < p.n_heads) {
+                    if (h0 + i < h_end) {
                         uint2 o2;
                         o2.x = pack_bf16(x[i].x * p.scale, x[i].y * p.scale);
                         o2.y = pack_bf16(x[i].z * p.scale, x[i].w * p.scale);
@@ -152,10 +154,10 @@ __global__ void __launch_bounds__(kPreThreads) zl_bwd_post_kernel(const BwdParam
                 float2 x[kBatch];
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i)
-                    if (h0 + i < p.n_heads) x[i] = __ldcs(reinterpret_cast<const float2*>(src + (int64_t)(h0 + i) * D));
+                    if (h0 + i < h_end) x[i] = __ldcs(reinterpret_cast<const float2*>(src + (int64_t)(h0 + i) * D));
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i)
-                    if (h0 + i < p.n_heads)
+                    if (h0 + i < h_end)
                         *reinterpret_cast<uint32_t*>(dst + (int64_t)(h0 + i) * D) = pack_bf16(x[i].x * p.scale, x[i].y * p.scale);
             }
         }

@@ -26,14 +26,21 @@ struct alignas(16) WorkItem {
     int32_t unit, head, row0, rows;
 };
 
-struct alignas(16) MergeGroup {
+// Shard tasks that share a query range and a head range; they are merged for heads
+// [head_begin, head_begin + head_count) only.
+struct alignas(32) MergeGroup {
     int32_t q_off, q_len;
     int32_t part_begin, n_parts;  // range in the merge part list (partial slot row offsets)
+    int32_t head_begin, head_count;
+    int32_t pad_[2];
 };
 
-// A distinct query range: rows [slot, slot + pad128(q_len)) of the backward scratch arrays.
-struct alignas(16) QGroup {
+// A distinct (query range, head range): rows [slot, slot + pad128(q_len)) of the backward scratch
+// arrays, of which only the heads of the range are used.
+struct alignas(32) QGroup {
     int32_t q_off, q_len, slot, pad;
+    int32_t head_begin, head_count;
+    int32_t pad_[2];
 };
 
 struct alignas(16) KvGroup {
@@ -41,10 +48,20 @@ struct alignas(16) KvGroup {
     int32_t task_begin, n_tasks;  // range in the kv-group task list
 };
 
+// One attention problem of a placement as the builder receives it: a whole sequence (q range ==
+// kv range, final after the forward launch) or a shard (one query chunk x one K/V chunk), over the
+// heads [head_begin, head_begin + head_count).
+struct InputTask {
+    int32_t q_off, q_len, kv_off, kv_len, seq_id;
+    int32_t head_begin, head_count;
+    int32_t shard_idx;  // index into the caller's shard array, -1 for a whole sequence
+};
+
 // Everything zl_build_tasks derives from a placement, on the host.
 struct Schedule {
     int32_t n_heads = 0, head_dim = 0, total_q = 0, total_kv = 0;
     std::vector<Task> tasks;
+    std::vector<int32_t> task_head_begin, task_head_count;  // per task (host only: items carry their head)
     std::vector<int32_t> shard_to_task;     // per input shard: task index or -1 (q_len == 0)
     std::vector<int32_t> shard_slot_off;    // per input shard: slot row offset (or 0)
     std::vector<int32_t> shard_slot_rows;   // per input shard: padded slot rows (0 if skipped)
@@ -65,10 +82,10 @@ struct Schedule {
 };
 
 // Validates the placement and fills `s`.  Pure host code, no CUDA.
-// `flags`: ZL_BUILD_* bits of zl_build_tasks_ex.
-zl_status build_schedule(const int32_t* cu_seqlens, int32_t n_whole, const zl_shard_desc* shards,
-                         int32_t n_shards, int32_t total_q, int32_t total_kv, int32_t n_heads,
-                         int32_t head_dim, uint32_t flags, Schedule* s);
+// `in`: whole sequences first (in placement order), then shards (in the caller's order); `n_shards` is
+// the size of the caller's shard array.  `flags`: ZL_BUILD_* bits of zl_build_tasks_ex.
+zl_status build_schedule(const std::vector<InputTask>& in, int32_t n_shards, int32_t total_q, int32_t total_kv,
+                         int32_t n_heads, int32_t head_dim, uint32_t flags, Schedule* s);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -73,6 +73,7 @@ __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeP
             if (p.row_prefix[mid] <= r) lo = mid; else hi = mid;
         }
         const MergeGroup g = p.groups[lo];
+        if (h < g.head_begin || h >= g.head_begin + g.head_count) continue;  // the group's tasks do not run this head
         const int row = (int)(r - p.row_prefix[lo]);
         float acc[V];
 #pragma unroll

@@ -199,3 +199,86 @@ def test_fusion_needs_contiguous_chunks_and_keeps_validation(Z):
     with pytest.raises(Z.ZlError) as e:
         Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, 1, 64, flags=2)
     assert e.value.status == 1           # unknown flag
+
+
+# --------------------------------------------------------------------------------------------------
+# Per-task head ranges (zl_build_tasks_heads)
+# --------------------------------------------------------------------------------------------------
+
+def _build_heads(Z, p, flags=0):
+    return Z.build_tasks_heads(p.whole_descs(), p.shards, p.shard_head_ranges(), p.total_q, p.total_kv,
+                               p.n_heads, p.head_dim, flags=flags)
+
+
+def test_heads_builder_with_full_ranges_equals_plain_builder(Z):
+    for ci in (1, 3):
+        p = W.config(ci)
+        a = _build(Z, p)
+        b = Z.build_tasks_heads(p.whole_descs(), p.shards, None, p.total_q, p.total_kv, p.n_heads, p.head_dim)
+        assert a.fwd_items() == b.fwd_items() and a.bwd_items() == b.bwd_items()
+        assert bytes(a.info) == bytes(b.info)
+        assert [a.partial_slot(i) for i in range(len(p.shards))] == [b.partial_slot(i) for i in range(len(p.shards))]
+
+
+def test_head_range_items_cover_each_task_on_its_heads_only(Z):
+    p = W.ulysses_mix_placement(n_heads=12, head_dim=128, n_images=6, image_len=1560, seq_len=3600, degree=2)
+    h = _build_heads(Z, p)
+    whole = p.whole_descs()
+    assert h.info.n_tasks == 8 and h.info.n_merge_groups == 0 and h.info.n_kv_groups == 8
+    seen = {}
+    for (t, hd, r0, rows) in h.fwd_items():
+        off, ln, hb, hc = whole[t]
+        assert hb <= hd < hb + hc, "work item on a head outside its task's range"
+        cov = seen.setdefault((t, hd), np.zeros(ln, dtype=int))
+        cov[r0:r0 + rows] += 1
+    assert len(seen) == sum(w[3] for w in whole) and all((c == 1).all() for c in seen.values())
+    # backward: the two sequences that share rows are two kv groups, six heads each
+    per_group = {}
+    for (g, hd, r0, rows) in h.bwd_items():
+        per_group.setdefault(g, set()).add(hd)
+    sizes = sorted(len(v) for v in per_group.values())
+    assert sizes == [6, 6] + [12] * 6
+    # counted work: 6 images x 12 heads + 2 sequences x 6 heads
+    assert p.fwd_flops() == 4.0 * 128 * (6 * 1560 ** 2 * 12 + 2 * 3600 ** 2 * 6)
+
+
+def test_head_range_shards_form_groups_per_head_range(Z):
+    # one query range served on heads [0,2) by two K/V chunks and on heads [2,4) by one chunk over the same rows
+    whole = [(0, 100, 0, 4)]
+    shards = [(100, 100, 100, 70, 0, 0, 2), (100, 100, 170, 80, 0, 0, 2), (100, 100, 100, 150, 1, 2, 2)]
+    p = W.head_range_placement("hr", 4, 64, 3, whole, shards, 200, 250)
+    h = _build_heads(Z, p)
+    assert h.info.n_tasks == 4 and h.info.n_merge_groups == 2 and h.info.n_kv_groups == 4
+    heads_of_task = {}
+    for (t, hd, r0, rows) in h.fwd_items():
+        heads_of_task.setdefault(t, set()).add(hd)
+    assert heads_of_task == {0: {0, 1, 2, 3}, 1: {0, 1}, 2: {0, 1}, 3: {2, 3}}
+    # with chunk fusion the two-chunk range becomes one final task; the single-chunk range stays a shard
+    hf = _build_heads(Z, p, flags=Z.BUILD_FUSE_LOCAL_CHUNKS)
+    assert hf.info.n_fused_ranges == 1 and hf.info.n_tasks == 3 and hf.info.n_merge_groups == 1
+
+
+def test_head_range_validation(Z):
+    def build(whole, shards, H=4, tq=300, tkv=300):
+        p = W.head_range_placement("v", H, 64, 0, whole, shards, tq, tkv)
+        return _build_heads(Z, p)
+
+    build([(0, 100, 0, 2), (0, 100, 2, 2)], [])                       # same rows, disjoint heads: fine
+    build([(0, 100, 0, 4), (100, 50, 1, 2)], [])                      # different rows, nested head ranges: fine
+    for whole, shards, status in [
+        ([(0, 100, 0, 3), (50, 100, 2, 2)], [], 2),                   # rows overlap on head 2
+        ([(0, 100, 0, 3), (0, 100, 2, 2)], [], 2),                    # identical rows, head ranges intersect but differ
+        ([(0, 100, 0, 2), (0, 100, 0, 2)], [], 2),                    # the same sequence twice
+        ([(0, 100, 0, 5)], [], 1),                                    # head range beyond n_heads
+        ([(0, 100, 2, 0)], [], 1),                                    # empty head range
+        ([(0, 100, -1, 2)], [], 1),
+        ([(0, 100, 0, 4)], [(100, 50, 100, 50, 0, 0, 2), (100, 50, 150, 50, 0, 1, 2)], 2),   # one query range, head ranges intersect but differ
+        ([(0, 100, 0, 4)], [(100, 50, 100, 50, 0, 0, 2), (150, 50, 100, 50, 0, 1, 2)], 2),   # one key range, same
+        ([(0, 100, 0, 4)], [(50, 50, 100, 50, 0, 0, 2)], 2),          # shard inside the whole region
+    ]:
+        with pytest.raises(Z.ZlError) as e:
+            build(whole, shards)
+        assert e.value.status == status, (whole, shards, e.value.status)
+    # the same token ranges on disjoint head ranges are independent tasks
+    h = build([(0, 100, 0, 4)], [(100, 50, 100, 50, 0, 0, 2), (100, 50, 100, 50, 0, 2, 2)])
+    assert h.info.n_tasks == 3 and h.info.n_merge_groups == 2

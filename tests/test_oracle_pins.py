@@ -403,6 +403,42 @@ def test_placement_backward_finite_differences_through_shard_and_merge():
         assert np.linalg.norm(fd - g[name]) / np.linalg.norm(g[name]) < 1e-7
 
 
+def test_head_range_placement_against_per_head_library_calls():
+    """Tasks over head ranges: each head of a row block belongs to the problems that list it, and only
+    to those.  Library routine + autograd per (problem, head); (row, head) pairs no problem covers get
+    no output and no gradient."""
+    whole = [(0, 5, 0, 3), (5, 9, 0, 1), (5, 9, 1, 2)]          # two sequences share rows 5..13 on disjoint heads
+    shards = [(14, 6, 14, 4, 0, 0, 2), (14, 6, 18, 7, 0, 0, 2), (14, 6, 14, 11, 1, 2, 1)]
+    p = W.head_range_placement("hr", 3, 8, 77, whole, shards, 20, 25)
+    probs = A.logical_problems(p)
+    assert [(x["q_off"], x["q_len"], x["heads"]) for x in probs] == \
+        [(0, 5, (0, 3)), (5, 9, (0, 1)), (5, 9, (1, 2)), (14, 6, (0, 2)), (14, 6, (2, 1))]
+    assert probs[3]["kv_ranges"] == [(14, 4), (18, 7)] and probs[4]["kv_ranges"] == [(14, 11)]
+    Q, K, V, dO = _tensors(p, np.random.RandomState(54))
+    out = A.placement_fwd(p, Q, K, V)
+    g = A.placement_bwd(p, Q, K, V, dO)
+    s = A.placement_bwd_shard_form(p, Q, K, V, dO)
+    tQ, tK, tV = (torch.from_numpy(x.copy()).requires_grad_(True) for x in (Q, K, V))
+    loss = 0
+    covered = np.zeros((p.total_q, p.n_heads), dtype=bool)
+    for (qo, ql, ko, kl, hb, hc) in [(0, 5, 0, 5, 0, 3), (5, 9, 5, 9, 0, 1), (5, 9, 5, 9, 1, 2),
+                                     (14, 6, 14, 11, 0, 2), (14, 6, 14, 11, 2, 1)]:
+        for h in range(hb, hb + hc):
+            Ot, lt = _torch_ref(Q[qo:qo + ql, h], K[ko:ko + kl, h], V[ko:ko + kl, h], p.scale)
+            np.testing.assert_allclose(out["O"][qo:qo + ql, h], Ot, atol=1e-13)
+            np.testing.assert_allclose(out["LSE"][h, qo:qo + ql], lt, atol=1e-13)
+            covered[qo:qo + ql, h] = True
+            o = torch.nn.functional.scaled_dot_product_attention(
+                tQ[qo:qo + ql, h][None], tK[ko:ko + kl, h][None], tV[ko:ko + kl, h][None], scale=p.scale)[0]
+            loss = loss + (o * torch.from_numpy(dO[qo:qo + ql, h])).sum()
+    loss.backward()
+    assert np.isnan(out["LSE"].T[~covered]).all() and not np.isnan(out["LSE"].T[covered]).any()
+    for name, ref in (("dQ", tQ.grad), ("dK", tK.grad), ("dV", tV.grad)):
+        np.testing.assert_allclose(g[name], ref.numpy(), atol=1e-12)
+        np.testing.assert_allclose(s[name], ref.numpy(), atol=1e-12)
+    assert np.all(g["dQ"][~covered] == 0)
+
+
 # ------------------------------------------------------------------ config 1: generator + library
 
 def _cfg1_tensors():

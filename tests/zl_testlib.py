@@ -55,7 +55,11 @@ class GpuRun:
         self.Z = Z
         self.p = p
         self.scale = p.scale if scale is None else scale
-        self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, p.n_heads, p.head_dim, flags=flags)
+        if p.has_head_ranges:
+            self.h = Z.build_tasks_heads(p.whole_descs(), p.shards, p.shard_head_ranges(), p.total_q, p.total_kv,
+                                         p.n_heads, p.head_dim, flags=flags)
+        else:
+            self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, p.n_heads, p.head_dim, flags=flags)
         self.info = self.h.info
 
     def forward(self, Q, K, V, merge=True):
@@ -90,30 +94,31 @@ class GpuRun:
 
 
 def covered_rows(p):
-    """Boolean masks of Q-space / KV-space rows covered by at least one task."""
-    q = np.zeros(p.total_q, dtype=bool)
-    kv = np.zeros(p.total_kv, dtype=bool)
-    for i in range(p.n_whole):
-        q[p.cu_seqlens[i]:p.cu_seqlens[i + 1]] = True
-        kv[p.cu_seqlens[i]:p.cu_seqlens[i + 1]] = True
-    for (qo, ql, ko, kl, _) in p.shards:
+    """Boolean masks [rows, H] of the (row, head) pairs of Q-space / KV-space covered by at least one task."""
+    q = np.zeros((p.total_q, p.n_heads), dtype=bool)
+    kv = np.zeros((p.total_kv, p.n_heads), dtype=bool)
+    for (o, l, hb, hc) in p.whole_descs():
+        q[o:o + l, hb:hb + hc] = True
+        kv[o:o + l, hb:hb + hc] = True
+    for (qo, ql, ko, kl, _), (hb, hc) in zip(p.shards, p.shard_head_ranges()):
         if ql > 0:
-            q[qo:qo + ql] = True
+            q[qo:qo + ql, hb:hb + hc] = True
             if kl > 0:
-                kv[ko:ko + kl] = True
+                kv[ko:ko + kl, hb:hb + hc] = True
     return q, kv
 
 
 def check_forward(p, O_gpu, LSE_gpu, ref, tol=(TOL_O_MAX, TOL_O_MEAN, TOL_LSE_MAX), heads=None):
-    """Compare GPU O/LSE (torch tensors) with oracle dict (placement_fwd) on covered rows."""
+    """Compare GPU O/LSE (torch tensors) with oracle dict (placement_fwd) on covered (row, head) pairs."""
     hs = list(range(p.n_heads)) if heads is None else list(heads)
-    qmask, _ = covered_rows(p)
+    qmask = covered_rows(p)[0][:, hs]                  # [rows, nh]
     Og = dev_to_f64(O_gpu)[:, hs, :]
-    Lg = dev_to_f64(LSE_gpu)[hs, :]
+    Lg = dev_to_f64(LSE_gpu)[hs, :].T                  # [rows, nh]
+    Lr = ref["LSE"].T
     eo = np.abs(Og[qmask] - ref["O"][qmask])
-    fin = np.isfinite(ref["LSE"][:, qmask])
-    el = np.abs(Lg[:, qmask][fin] - ref["LSE"][:, qmask][fin])
-    assert np.array_equal(np.isneginf(Lg[:, qmask]), np.isneginf(ref["LSE"][:, qmask]))
+    fin = np.isfinite(Lr[qmask])
+    el = np.abs(Lg[qmask][fin] - Lr[qmask][fin])
+    assert np.array_equal(np.isneginf(Lg[qmask]), np.isneginf(Lr[qmask]))
     # error beyond the unavoidable bf16 rounding of the output (half an ulp = 2^-9 relative)
     excess = eo - np.abs(ref["O"][qmask]) * 2.0 ** -8
     stats = dict(o_max=float(eo.max()) if eo.size else 0.0, o_mean=float(eo.mean()) if eo.size else 0.0,
@@ -122,9 +127,9 @@ def check_forward(p, O_gpu, LSE_gpu, ref, tol=(TOL_O_MAX, TOL_O_MEAN, TOL_LSE_MA
     assert stats["o_max"] <= tol[0], stats
     assert stats["o_mean"] <= tol[1], stats
     assert stats["lse_max"] <= tol[2], stats
-    # rows outside every task keep the sentinel
+    # (row, head) pairs outside every task keep the sentinel
     if (~qmask).any():
-        assert np.all(Og[~qmask] == SENTINEL) and np.all(Lg[:, ~qmask] == SENTINEL)
+        assert np.all(Og[~qmask] == SENTINEL) and np.all(Lg[~qmask] == SENTINEL)
     return stats
 
 
@@ -148,12 +153,12 @@ def check_backward(p, dQ, dK, dV, ref, tol=TOL_GRAD_REL, heads=None, row_tol=TOL
     hs = list(range(p.n_heads)) if heads is None else list(heads)
     qmask, kvmask = covered_rows(p)
     out = {}
-    for name, g, mask in (("dQ", dQ, qmask), ("dK", dK, kvmask), ("dV", dV, kvmask)):
+    for name, g, mask in (("dQ", dQ, qmask[:, hs]), ("dK", dK, kvmask[:, hs]), ("dV", dV, kvmask[:, hs])):
         gg = dev_to_f64(g)[:, hs, :]
         out[name] = rel_fro(gg[mask], ref[name][mask])
         assert out[name] <= tol, (name, out)
         out[name + "_row"] = row_rel(gg[mask], ref[name][mask])
         assert out[name + "_row"] <= row_tol, (name, "row-wise", out)
         if (~mask).any():
-            assert np.all(gg[~mask] == SENTINEL), f"{name}: rows outside every task were written"
+            assert np.all(gg[~mask] == SENTINEL), f"{name}: (row, head) pairs outside every task were written"
     return out

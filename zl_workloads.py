@@ -40,6 +40,12 @@ class Placement:
     shards: Tuple[Tuple[int, int, int, int, int], ...]
     total_q: int
     total_kv: int
+    # Head ranges (Ulysses-shaped tasks: all tokens of a sequence for a subset of the heads).  None = every
+    # task covers all heads.  With `whole_ranges` the whole sequences are given as (off, len) pairs instead
+    # of cu_seqlens, which lets two sequences own the same rows on disjoint head ranges.
+    whole_heads: Optional[Tuple[Tuple[int, int], ...]] = None   # (head_begin, head_count) per whole sequence
+    shard_heads: Optional[Tuple[Tuple[int, int], ...]] = None   # (head_begin, head_count) per shard
+    whole_ranges: Optional[Tuple[Tuple[int, int], ...]] = None  # (off, len) per whole sequence
 
     @property
     def scale(self) -> float:
@@ -47,20 +53,40 @@ class Placement:
 
     @property
     def n_whole(self) -> int:
-        return len(self.cu_seqlens) - 1
+        return len(self.whole_ranges) if self.whole_ranges is not None else len(self.cu_seqlens) - 1
+
+    @property
+    def has_head_ranges(self) -> bool:
+        return self.whole_heads is not None or self.shard_heads is not None or self.whole_ranges is not None
+
+    def whole_descs(self) -> List[Tuple[int, int, int, int]]:
+        """(off, len, head_begin, head_count) per whole sequence."""
+        rng = self.whole_ranges if self.whole_ranges is not None else \
+            [(self.cu_seqlens[i], self.cu_seqlens[i + 1] - self.cu_seqlens[i]) for i in range(len(self.cu_seqlens) - 1)]
+        hd = self.whole_heads if self.whole_heads is not None else [(0, self.n_heads)] * len(rng)
+        assert len(hd) == len(rng)
+        return [(int(o), int(l), int(hb), int(hc)) for (o, l), (hb, hc) in zip(rng, hd)]
+
+    def shard_head_ranges(self) -> List[Tuple[int, int]]:
+        if self.shard_heads is None:
+            return [(0, self.n_heads)] * len(self.shards)
+        assert len(self.shard_heads) == len(self.shards)
+        return [(int(a), int(b)) for a, b in self.shard_heads]
 
     def whole_lengths(self) -> List[int]:
-        return [self.cu_seqlens[i + 1] - self.cu_seqlens[i] for i in range(self.n_whole)]
+        return [w[1] for w in self.whole_descs()]
 
     def pairs_per_head(self) -> int:
-        """Number of (query, key) score elements per head over all tasks."""
+        """Number of (query, key) score elements per head over all tasks (all-head placements)."""
         n = sum(l * l for l in self.whole_lengths())
         n += sum(s[1] * s[3] for s in self.shards)
         return n
 
     def fwd_flops(self) -> float:
-        """Counted forward FLOPs: 4 * Lq * Lkv * d * H summed over tasks."""
-        return 4.0 * self.pairs_per_head() * self.head_dim * self.n_heads
+        """Counted forward FLOPs: 4 * Lq * Lkv * d * (heads of the task) summed over tasks."""
+        pairs = sum(l * l * hc for (_, l, _, hc) in self.whole_descs())
+        pairs += sum(s[1] * s[3] * hc for s, (_, hc) in zip(self.shards, self.shard_head_ranges()))
+        return 4.0 * pairs * self.head_dim
 
     def bwd_flops(self) -> float:
         return 2.5 * self.fwd_flops()
@@ -225,3 +251,29 @@ def custom_placement(name: str, n_heads: int, head_dim: int, seed: int,
                      total_q: int, total_kv: int) -> Placement:
     return Placement(name, n_heads, head_dim, seed, tuple(int(c) for c in cu_seqlens),
                      tuple(tuple(int(v) for v in s) for s in shards), int(total_q), int(total_kv))
+
+
+def head_range_placement(name: str, n_heads: int, head_dim: int, seed: int,
+                         whole: Sequence[Sequence[int]], shards: Sequence[Sequence[int]],
+                         total_q: int, total_kv: int) -> Placement:
+    """A placement whose tasks cover head ranges: `whole` holds (off, len, head_begin, head_count) per
+    whole sequence, `shards` holds (q_off, q_len, kv_off, kv_len, seq_id, head_begin, head_count)."""
+    return Placement(name, n_heads, head_dim, seed, (0,),
+                     tuple(tuple(int(v) for v in s[:5]) for s in shards), int(total_q), int(total_kv),
+                     whole_heads=tuple((int(w[2]), int(w[3])) for w in whole),
+                     shard_heads=tuple((int(s[5]), int(s[6])) for s in shards),
+                     whole_ranges=tuple((int(w[0]), int(w[1])) for w in whole))
+
+
+def ulysses_mix_placement(n_heads: int = 12, head_dim: int = 128, seed: int = 21, n_images: int = 6,
+                          image_len: int = 1560, seq_len: int = 3600, degree: int = 2) -> Placement:
+    """Whole images over all heads next to `degree` Ulysses-shaped sequences, each holding all of its
+    `seq_len` tokens for n_heads / degree heads; the Ulysses sequences share one block of rows, side by
+    side in the head dimension (the layout a QKV-packed all-to-all over `degree` ranks delivers)."""
+    assert n_heads % degree == 0
+    hc = n_heads // degree
+    whole = [(i * image_len, image_len, 0, n_heads) for i in range(n_images)]
+    base = n_images * image_len
+    whole += [(base, seq_len, r * hc, hc) for r in range(degree)]
+    total = base + seq_len
+    return head_range_placement("ulysses_mix", n_heads, head_dim, seed, whole, [], total, total)
