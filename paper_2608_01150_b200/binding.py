@@ -96,6 +96,8 @@ def _load():
     lib.zl_get_kernel_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.zl_debug_set_fwd_order.restype = ctypes.c_int
     lib.zl_debug_set_fwd_order.argtypes = [vp, i32, vp]
+    lib.zl_set_bwd_kernel.restype = ctypes.c_int
+    lib.zl_set_bwd_kernel.argtypes = [vp, i32]
     lib.zl_selftest_bounded_wait.restype = ctypes.c_int
     lib.zl_selftest_bounded_wait.argtypes = [vp, i32, vp]
     lib.zl_status_str.restype = ctypes.c_char_p
@@ -186,6 +188,10 @@ class TaskHandle:
     def set_fwd_order(self, mode: int, stream=None):
         """0 longest-first (default), 1 placement order, 2 shortest-first (measurement aid)."""
         _check(_lib.zl_debug_set_fwd_order(self._ptr, mode, _stream_ptr(stream)), "zl_debug_set_fwd_order")
+
+    def set_bwd_kernel(self, kernel: int):
+        """0 library default, 1 one CTA per key tile, 2 CTA pairs (head_dim 128)."""
+        _check(_lib.zl_set_bwd_kernel(self._ptr, kernel), "zl_set_bwd_kernel")
 
     def selftest_bounded_wait(self, limit_us: int = 1000, stream=None):
         """Launches a kernel whose bounded wait must expire; read the outcome with last_device_status()."""

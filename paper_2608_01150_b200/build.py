@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 LIB = os.path.join(_PKG, "libzellige.so")
-SOURCES = ["zl_api.cu", "zl_fwd.cu", "zl_merge.cu", "zl_bwd.cu", "zl_tasks.cpp"]
+SOURCES = ["zl_api.cu", "zl_fwd.cu", "zl_merge.cu", "zl_bwd.cu", "zl_bwd_pair.cu", "zl_tasks.cpp"]
 
 
 def _sources():

@@ -23,6 +23,8 @@ struct zl_tasks {
     Task* d_tasks = nullptr;
     WorkItem* d_fwd_items = nullptr;
     WorkItem* d_bwd_items = nullptr;
+    WorkItem* d_bwd_pair_items = nullptr;
+    int bwd_kernel = 0;           // 0: library default, 1: one CTA per key tile, 2: CTA pairs (head_dim 128)
     MergeGroup* d_merge_groups = nullptr;
     int32_t* d_merge_parts = nullptr;
     int32_t* d_merge_prefix = nullptr;
@@ -76,6 +78,7 @@ bool make_tmap(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int 
 }
 
 constexpr int kMaxTimedLaunches = 1024;
+constexpr bool kDefaultBwdPair = false;  // which backward main kernel a handle uses unless zl_set_bwd_kernel chose one
 
 // Brackets one kernel launch with events when timing is enabled on the handle.
 struct LaunchTimer {
@@ -99,16 +102,33 @@ struct LaunchTimer {
     ~LaunchTimer() { if (stop) cudaEventRecord(stop, cs); }
 };
 
-// Tensor map over the fp32 dQ accumulator [rows, H, d]: box = 32 columns x 1 head x 128 rows.
-bool make_tmap_f32_acc(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim, int box_rows = 32) {
+// Tensor map over the fp32 dQ accumulator [rows, H, d]: box = 32 columns x 1 head x box_rows rows with 128-byte
+// swizzle, or (box_cols = 16) 16 columns with 64-byte swizzle.
+bool make_tmap_f32_acc(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int head_dim, int box_rows = 32,
+                       int box_cols = 32) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)(rows > 0 ? rows : 1)};
     cuuint64_t strides[2] = {(cuuint64_t)head_dim * 4, (cuuint64_t)head_dim * 4 * n_heads};
-    cuuint32_t box[3] = {32, 1, (cuuint32_t)box_rows};  // 32 fp32 columns x one warp's 32 rows (dQ) or a 128-row tile
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, 1, (cuuint32_t)box_rows};  // one warp's 32 rows (dQ) or a 128-row tile
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, box_cols == 16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// The augmentation tiles of the backward workspace as a 2-D array of 1 KB rows (256 x 32-bit): row
+// tile * 4 + chunk * 2 + half holds one K chunk of one 64-row half of a tile.
+bool make_tmap_aug_rows(CUtensorMap* m, const void* base, int64_t n_tiles) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {256, (cuuint64_t)(n_tiles > 0 ? n_tiles * 4 : 1)};
+    cuuint64_t strides[1] = {1024};
+    cuuint32_t box[2] = {256, 1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -218,6 +238,7 @@ zl_status zl_build_tasks_heads(const zl_whole_desc* whole, int32_t n_whole, cons
     const size_t o_tasks = place<Task>(off, s.tasks.size());
     const size_t o_fwd = place<WorkItem>(off, s.fwd_items.size());
     const size_t o_bwd = place<WorkItem>(off, s.bwd_items.size());
+    const size_t o_bwd2 = place<WorkItem>(off, s.bwd_pair_items.size());
     const size_t o_mg = place<MergeGroup>(off, s.merge_groups.size());
     const size_t o_mp = place<int32_t>(off, s.merge_parts.size());
     const size_t o_mr = place<int32_t>(off, s.merge_row_prefix.size());
@@ -232,6 +253,7 @@ zl_status zl_build_tasks_heads(const zl_whole_desc* whole, int32_t n_whole, cons
     put(o_tasks, s.tasks.data(), s.tasks.size() * sizeof(Task));
     put(o_fwd, s.fwd_items.data(), s.fwd_items.size() * sizeof(WorkItem));
     put(o_bwd, s.bwd_items.data(), s.bwd_items.size() * sizeof(WorkItem));
+    put(o_bwd2, s.bwd_pair_items.data(), s.bwd_pair_items.size() * sizeof(WorkItem));
     put(o_mg, s.merge_groups.data(), s.merge_groups.size() * sizeof(MergeGroup));
     put(o_mp, s.merge_parts.data(), s.merge_parts.size() * sizeof(int32_t));
     put(o_mr, s.merge_row_prefix.data(), s.merge_row_prefix.size() * sizeof(int32_t));
@@ -249,6 +271,7 @@ zl_status zl_build_tasks_heads(const zl_whole_desc* whole, int32_t n_whole, cons
     h->d_tasks = reinterpret_cast<Task*>(h->d_tables + o_tasks);
     h->d_fwd_items = reinterpret_cast<WorkItem*>(h->d_tables + o_fwd);
     h->d_bwd_items = reinterpret_cast<WorkItem*>(h->d_tables + o_bwd);
+    h->d_bwd_pair_items = reinterpret_cast<WorkItem*>(h->d_tables + o_bwd2);
     h->d_merge_groups = reinterpret_cast<MergeGroup*>(h->d_tables + o_mg);
     h->d_merge_parts = reinterpret_cast<int32_t*>(h->d_tables + o_mp);
     h->d_merge_prefix = reinterpret_cast<int32_t*>(h->d_tables + o_mr);
@@ -480,7 +503,22 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
         if (launch_bwd_pre(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
     }
     g_launches.fetch_add(1);
-    if (p.n_items > 0) {
+    const bool pair = s.head_dim == 128 && (t->bwd_kernel == 2 || (t->bwd_kernel == 0 && kDefaultBwdPair));
+    if (p.n_items > 0 && pair) {
+        CUtensorMap tq64, tdo64, taug, tdq16;
+        if (!make_tmap_f32_acc(&tdq16, ws + s.ws_dq_acc_off, s.q_pad_total, s.n_heads, s.head_dim, 32, 16) ||
+            !make_tmap(&tq64, q, s.total_q, s.n_heads, s.head_dim, 64, in_stride) ||
+            !make_tmap(&tdo64, d_o, s.total_q, s.n_heads, s.head_dim, 64, hd) ||
+            !make_tmap_aug_rows(&taug, p.aug, (s.q_pad_total / kTileQ) * s.n_heads))
+            return ZL_ERR_CUDA;
+        BwdParams pp = p;
+        pp.items = t->d_bwd_pair_items;
+        pp.n_items = (int32_t)s.bwd_pair_items.size();
+        const int n_clusters = std::min<int>(t->n_sms / 2, pp.n_items);
+        LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
+        if (launch_bwd_pair(tq, tq64, tk, tv, tdo, tdo64, tdq16, taug, pp, n_clusters, cs) != cudaSuccess) return ZL_ERR_CUDA;
+        g_launches.fetch_add(1);
+    } else if (p.n_items > 0) {
         const int grid = std::min<int>(t->n_sms, p.n_items);
         LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
         if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, tdq, tdk, tdv, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
@@ -579,6 +617,13 @@ zl_status zl_debug_set_fwd_order(zl_tasks* t, int32_t mode, void* stream) {
                         cudaMemcpyHostToDevice, cs) != cudaSuccess ||
         cudaStreamSynchronize(cs) != cudaSuccess)
         return ZL_ERR_CUDA;
+    return ZL_OK;
+}
+
+zl_status zl_set_bwd_kernel(zl_tasks* t, int32_t kernel) {
+    if (!t || kernel < 0 || kernel > 2) return ZL_ERR_INVALID_ARG;
+    if (kernel == 2 && t->sched.head_dim != 128) return ZL_ERR_UNSUPPORTED;
+    t->bwd_kernel = kernel;
     return ZL_OK;
 }
 

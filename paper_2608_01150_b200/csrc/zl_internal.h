@@ -74,6 +74,7 @@ struct Schedule {
     std::vector<int32_t> kv_group_tasks;
     std::vector<WorkItem> fwd_items;
     std::vector<WorkItem> bwd_items;
+    std::vector<WorkItem> bwd_pair_items;   // (kv group, head, first key row, rows <= 256): two key tiles per CTA pair
     int64_t partial_rows = 0;
     int32_t n_fused_ranges = 0;             // shard query ranges lowered to one final task (chunk fusion)
     size_t bwd_workspace_bytes = 0;

@@ -279,11 +279,20 @@ zl_status build_schedule(const std::vector<InputTask>& in, int32_t n_shards, int
             for (int32_t r = 0; r < s->kv_groups[g].kv_len; r += kTileKV)
                 s->bwd_items.push_back({(int32_t)g, h, r, std::min(kTileKV, s->kv_groups[g].kv_len - r)});
     }
-    std::stable_sort(s->bwd_items.begin(), s->bwd_items.end(), [&](const WorkItem& a, const WorkItem& b) {
+    auto bwd_order = [&](const WorkItem& a, const WorkItem& b) {
         if (group_cost[a.unit] != group_cost[b.unit]) return group_cost[a.unit] > group_cost[b.unit];
         if (a.rows != b.rows) return a.rows > b.rows;
         return std::tie(a.unit, a.head, a.row0) < std::tie(b.unit, b.head, b.row0);
-    });
+    };
+    std::stable_sort(s->bwd_items.begin(), s->bwd_items.end(), bwd_order);
+    // the same list in units of two key tiles, for the CTA-pair form of the main kernel
+    for (size_t g = 0; g < s->kv_groups.size(); ++g) {
+        const int32_t t0 = s->kv_group_tasks[s->kv_groups[g].task_begin];
+        for (int32_t h = s->task_head_begin[t0]; h < s->task_head_begin[t0] + s->task_head_count[t0]; ++h)
+            for (int32_t r = 0; r < s->kv_groups[g].kv_len; r += 2 * kTileKV)
+                s->bwd_pair_items.push_back({(int32_t)g, h, r, std::min(2 * kTileKV, s->kv_groups[g].kv_len - r)});
+    }
+    std::stable_sort(s->bwd_pair_items.begin(), s->bwd_pair_items.end(), bwd_order);
 
     // backward workspace over the padded query slots: fp32 dQ accumulator [q_pad, H, d], then one
     // 4 KB "augmentation" tile per (head, 128-row query tile) holding -LSE/scale and -D split

@@ -61,6 +61,11 @@ class GpuRun:
         else:
             self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, p.n_heads, p.head_dim, flags=flags)
         self.info = self.h.info
+        # ZL_TEST_BWD_KERNEL=1|2 runs the whole suite on one of the two backward main kernels
+        import os
+        k = int(os.environ.get("ZL_TEST_BWD_KERNEL", "0"))
+        if k == 1 or (k == 2 and p.head_dim == 128):
+            self.h.set_bwd_kernel(k)
 
     def forward(self, Q, K, V, merge=True):
         p, H, d = self.p, self.p.n_heads, self.p.head_dim
