@@ -136,7 +136,7 @@ def aggregate_tflops(world: int, flops_per_rank: float, ms_per_step: float) -> f
 class Workload:
     """Device tensors + task handle of one placement."""
 
-    def __init__(self, p, device, seed_shift=0, flags=0):
+    def __init__(self, p, device, seed_shift=0, flags=0, bwd_kernel=0):
         import torch
         import paper_2608_01150_b200 as Z
         import zl_workloads as W
@@ -147,6 +147,8 @@ class Workload:
         t0 = time.perf_counter()
         self.h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, H, d, flags=flags)
         self.build_ms = (time.perf_counter() - t0) * 1e3
+        if bwd_kernel and not (bwd_kernel == 2 and d != 128):
+            self.h.set_bwd_kernel(bwd_kernel)
         info = self.h.info
         self.O = torch.empty_like(self.Q)
         self.LSE = torch.empty(H, p.total_q, dtype=torch.float32, device=device)
@@ -314,7 +316,7 @@ def run_ours(args):
     peaks, peak_kind = load_peaks()
 
     p = W.config(args.config)
-    wl = Workload(p, device, seed_shift=rank * 7, flags=1 if args.fuse_local_chunks else 0)
+    wl = Workload(p, device, seed_shift=rank * 7, flags=1 if args.fuse_local_chunks else 0, bwd_kernel=args.bwd_kernel)
     K, Wm = args.steps, max(3, args.warmup)
     for _ in range(Wm):
         wl.step()
@@ -421,7 +423,7 @@ def run_ours(args):
         for ci in [int(x) for x in args.extra_configs.split(",") if x]:
             try:
                 pe = W.config(ci)
-                we = Workload(pe, device)
+                we = Workload(pe, device, bwd_kernel=args.bwd_kernel)
                 n = 3 if ci == 5 else 5
                 for _ in range(3):
                     we.step()
@@ -543,6 +545,61 @@ def run_ablation(args):
     print(json.dumps(out), flush=True)
 
 
+def run_cp(args):
+    """Context-parallel mode (not the headline): all N ranks share one 75,600-token video under N-way all-gather
+    context parallelism (Table II, configuration (q,1,1)) and each also runs six whole 1560-token images; one
+    layer forward + backward through the executor (K/V all-gather into local buffers -> one coalesced launch +
+    merge -> backward -> dK/dV reduce-scatter).  value = counted FLOPs of the whole job / slowest rank's time."""
+    import torch
+    import torch.distributed as dist
+    from paper_2608_01150_b200 import executor as E
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    else:
+        dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{29500 + os.getpid() % 2000}", rank=0, world_size=1)
+    H, d, L = 40, 128, 75600
+    segs = [E.Segment(0, L, (world, 1, 1), tuple(range(world)))] if world > 1 else [E.Segment(0, L // 8, (1, 1, 1), (0,))]
+    sid = 1
+    for r in range(world):
+        for _ in range(6):
+            segs.append(E.Segment(sid, 1560, (1, 1, 1), (r,)))
+            sid += 1
+    ex = E.CPExecutor(segs, H, d)
+    eng = E.EngineAttention(d)
+    T = ex.schedule.own_tokens
+    g = torch.Generator(device=device); g.manual_seed(7 + rank)
+    q, k, v, do = (torch.randn((T, H, d), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16) for _ in range(4))
+
+    def step():
+        ex.forward(q, k, v, eng.fwd)
+        ex.backward(do, eng.bwd)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize(); dist.barrier(); torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record(); torch.cuda.synchronize()
+    ms = reduce_max_ms(e0.elapsed_time(e1), dist, device) / args.steps
+    video_len = L if world > 1 else L // 8
+    pairs = video_len * video_len + world * 6 * 1560 * 1560
+    flops = 3.5 * 4.0 * pairs * d * H
+    if rank == 0:
+        print(json.dumps({"mode": "cp", "metric": METRIC, "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                          "n_gpus": world, "steps": args.steps, "ms_per_step": ms, "scaling": "strong (video) + weak (images)",
+                          "config": {"workload": f"one {video_len}-token video under {world}-way all-gather CP + 6 images per rank",
+                                     "n_heads": H, "head_dim": d, "collectives": [list(map(str, e)) for e in ex.log]}}), flush=True)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -555,6 +612,11 @@ def main():
     ap.add_argument("--fuse-local-chunks", action="store_true",
                     help="build the handle with ZL_BUILD_FUSE_LOCAL_CHUNKS: query ranges whose chunks are contiguous run "
                          "as one final task (no partials, nothing to merge); off by default")
+    ap.add_argument("--cp", action="store_true",
+                    help="context-parallel mode: one video under N-way all-gather CP across the N ranks + images per rank, "
+                         "through the executor (printed as its own JSON line, not the headline)")
+    ap.add_argument("--bwd-kernel", type=int, default=0, choices=[0, 1, 2],
+                    help="backward main kernel: 0 library default, 1 one CTA per key tile, 2 CTA pairs")
     ap.add_argument("--ablation", default="", choices=["", "straggler", "coalescing"],
                     help="print an extra measurement instead of the benchmark line")
     args = ap.parse_args()
@@ -566,11 +628,17 @@ def main():
     if args.impl == "reference":
         run_reference(args)
         return
+    if args.cp and (args.gpus == 1 or "WORLD_SIZE" in os.environ):
+        run_cp(args)
+        return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         port = 29500 + (os.getpid() % 2000)
         cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
                "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
         sys.exit(subprocess.call(cmd))
+    if args.cp:
+        run_cp(args)
+        return
     run_ours(args)
 
 
