@@ -15,32 +15,74 @@ namespace {
 
 constexpr int kMergeThreads = 256;
 
-// Up to NP parts: the parts' LSEs are read once and kept in registers (weights e_t / z).
+constexpr int kHeadsPerUnit = 4;  // a warp merges this many heads of one query row before it looks up the next row
+
+// One (row, head): LSE = M + log sum_t exp(LSE_t - M), O = sum_t exp(LSE_t - LSE) O_t in ascending part order.
+// NP > 0: at most NP parts, whose LSEs are read once and kept in registers (weights e_t / z); when the group has
+// exactly NP parts (the common case: one part per context-parallel chunk) all NP vector loads of the partial
+// outputs are issued before the first use, so a warp keeps NP x 512 bytes in flight.  NP = 0: any number of
+// parts, three passes over the parts' LSEs.
+// `src0` points at this lane's floats of part row 0, head h; `lse_h` at lse_partial[h][row]; `slot` holds the
+// parts' slot offsets (rows).
 template <int D, int NP>
-__device__ __forceinline__ float merge_small(const MergeParams& p, const MergeGroup& g, int row, int h, int lane,
-                                             float (&acc)[D / 32]) {
+__device__ __forceinline__ float merge_one(const MergeParams& p, const MergeGroup& g, const int32_t* part,
+                                           const int32_t (&slot)[NP > 0 ? NP : 1], const float* src0, const float* lse_h,
+                                           float (&acc)[D / 32]) {
     constexpr int V = D / 32;
-    const float* lse_h = p.lse_partial + (int64_t)h * p.partial_rows + row;
-    const int32_t* part = p.parts + g.part_begin;
-    float lt[NP];
-    float M = -INFINITY;
+    const int64_t part_stride = (int64_t)p.n_heads * D;  // floats between consecutive rows of o_partial
+    if constexpr (NP > 0) {
+        const bool all_parts = g.n_parts == NP;  // warp-uniform
+        float4 x4[NP];
+        float2 x2[NP];
+        if (all_parts) {
 #pragma unroll
-    for (int t = 0; t < NP; ++t) {
-        lt[t] = (t < g.n_parts) ? __ldg(lse_h + part[t]) : -INFINITY;
-        M = fmaxf(M, lt[t]);
-    }
-    float z = 0.f;
+            for (int t = 0; t < NP; ++t) {
+                const float* src = src0 + slot[t] * part_stride;
+                if constexpr (V == 4) x4[t] = __ldcs(reinterpret_cast<const float4*>(src));
+                else x2[t] = __ldcs(reinterpret_cast<const float2*>(src));
+            }
+        }
+        float lt[NP];
+        float M = -INFINITY;
 #pragma unroll
-    for (int t = 0; t < NP; ++t) {
-        lt[t] = (M == -INFINITY) ? 0.f : __expf(lt[t] - M);  // 0 for absent parts
-        z += lt[t];
-    }
-    const float inv_z = (z > 0.f) ? 1.f / z : 0.f;
+        for (int t = 0; t < NP; ++t) {
+            lt[t] = (t < g.n_parts) ? __ldg(lse_h + slot[t]) : -INFINITY;
+            M = fmaxf(M, lt[t]);
+        }
+        float z = 0.f;
 #pragma unroll
-    for (int t = 0; t < NP; ++t) {
-        if (t < g.n_parts) {
-            const float w = lt[t] * inv_z;
-            const float* src = p.o_partial + (((int64_t)part[t] + row) * p.n_heads + h) * D + lane * V;
+        for (int t = 0; t < NP; ++t) {
+            lt[t] = (M == -INFINITY) ? 0.f : __expf(lt[t] - M);  // 0 for absent parts
+            z += lt[t];
+        }
+        const float inv_z = (z > 0.f) ? 1.f / z : 0.f;
+#pragma unroll
+        for (int t = 0; t < NP; ++t) {
+            if (t < g.n_parts) {
+                const float w = lt[t] * inv_z;
+                if (!all_parts) {
+                    const float* src = src0 + slot[t] * part_stride;
+                    if constexpr (V == 4) x4[t] = __ldcs(reinterpret_cast<const float4*>(src));
+                    else x2[t] = __ldcs(reinterpret_cast<const float2*>(src));
+                }
+                if constexpr (V == 4) {
+                    acc[0] = fmaf(w, x4[t].x, acc[0]); acc[1] = fmaf(w, x4[t].y, acc[1]);
+                    acc[2] = fmaf(w, x4[t].z, acc[2]); acc[3] = fmaf(w, x4[t].w, acc[3]);
+                } else {
+                    acc[0] = fmaf(w, x2[t].x, acc[0]); acc[1] = fmaf(w, x2[t].y, acc[1]);
+                }
+            }
+        }
+        return (M == -INFINITY) ? -INFINITY : M + logf(z);
+    } else {
+        float M = -INFINITY;
+        for (int t = 0; t < g.n_parts; ++t) M = fmaxf(M, __ldg(lse_h + part[t]));
+        float z = 0.f;
+        for (int t = 0; t < g.n_parts; ++t) z += (M == -INFINITY) ? 0.f : __expf(__ldg(lse_h + part[t]) - M);
+        const float L = (M == -INFINITY) ? -INFINITY : M + logf(z);
+        for (int t = 0; t < g.n_parts; ++t) {
+            const float w = (L == -INFINITY) ? 0.f : __expf(__ldg(lse_h + part[t]) - L);
+            const float* src = src0 + part[t] * part_stride;
             if constexpr (V == 4) {
                 const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
                 acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
@@ -50,22 +92,25 @@ __device__ __forceinline__ float merge_small(const MergeParams& p, const MergeGr
                 acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
             }
         }
+        return L;
     }
-    return (M == -INFINITY) ? -INFINITY : M + logf(z);
 }
 
 // NP = 4 or 8: every group has at most NP parts (chosen by the launcher); NP = 0: any number of parts.
+// A unit of work is one query row and kHeadsPerUnit consecutive heads: the group lookup, the parts' slots and
+// the row's base addresses are worked out once per unit (the kernel is bound by instruction issue, not by DRAM).
 template <int D, int NP>
-__global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeParams p) {  // 8 blocks = 64 warps per SM
+__global__ void __launch_bounds__(kMergeThreads, NP == 8 ? 3 : (NP == 4 ? 4 : 8)) zl_merge_kernel(const MergeParams p) {
     constexpr int V = D / 32;  // floats per lane: 4 (d=128) or 2 (d=64)
     const int lane = threadIdx.x & 31;
     const int warps_per_block = kMergeThreads / 32;
     const int64_t n_rows = p.row_prefix[p.n_groups];
-    const int64_t n_units = n_rows * p.n_heads;
+    const int head_chunks = (p.n_heads + kHeadsPerUnit - 1) / kHeadsPerUnit;
+    const int64_t n_units = n_rows * head_chunks;
     for (int64_t u = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); u < n_units;
          u += (int64_t)gridDim.x * warps_per_block) {
-        const int64_t r = u / p.n_heads;
-        const int h = (int)(u - r * p.n_heads);
+        const int64_t r = u / head_chunks;
+        const int hc = (int)(u - r * head_chunks);
         // group of flat row r: binary search over the prefix sums
         int lo = 0, hi = p.n_groups;
         while (hi - lo > 1) {
@@ -73,56 +118,37 @@ __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeP
             if (p.row_prefix[mid] <= r) lo = mid; else hi = mid;
         }
         const MergeGroup g = p.groups[lo];
-        if (h < g.head_begin || h >= g.head_begin + g.head_count) continue;  // the group's tasks do not run this head
+        const int h_begin = max(hc * kHeadsPerUnit, g.head_begin);   // heads outside the group's range: no task runs them
+        const int h_end = min(min((hc + 1) * kHeadsPerUnit, p.n_heads), g.head_begin + g.head_count);
+        if (h_begin >= h_end) continue;
         const int row = (int)(r - p.row_prefix[lo]);
-        float acc[V];
-#pragma unroll
-        for (int i = 0; i < V; ++i) acc[i] = 0.f;
-        float L;
+        const int32_t* part = p.parts + g.part_begin;
+        int32_t slot[NP > 0 ? NP : 1];
         if constexpr (NP > 0) {
-            L = merge_small<D, NP>(p, g, row, h, lane, acc);
-        } else {
-            // any number of parts: three passes over the parts' LSEs
-            float M = -INFINITY;
-            for (int t = 0; t < g.n_parts; ++t) {
-                const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
-                M = fmaxf(M, __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr));
-            }
-            float z = 0.f;
-            for (int t = 0; t < g.n_parts; ++t) {
-                const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
-                const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
-                z += (M == -INFINITY) ? 0.f : __expf(lt - M);
-            }
-            L = (M == -INFINITY) ? -INFINITY : M + logf(z);
-            for (int t = 0; t < g.n_parts; ++t) {
-                const int64_t pr = (int64_t)p.parts[g.part_begin + t] + row;
-                const float lt = __ldg(p.lse_partial + (int64_t)h * p.partial_rows + pr);
-                const float w = (L == -INFINITY) ? 0.f : __expf(lt - L);
-                const float* src = p.o_partial + (pr * p.n_heads + h) * D + lane * V;
-                if constexpr (V == 4) {
-                    const float4 x = __ldcs(reinterpret_cast<const float4*>(src));
-                    acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
-                    acc[2] = fmaf(w, x.z, acc[2]); acc[3] = fmaf(w, x.w, acc[3]);
-                } else {
-                    const float2 x = __ldcs(reinterpret_cast<const float2*>(src));
-                    acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
-                }
-            }
+#pragma unroll
+            for (int t = 0; t < NP; ++t) slot[t] = (t < g.n_parts) ? __ldg(part + t) : 0;
         }
         const int64_t qrow = (int64_t)g.q_off + row;
-        __nv_bfloat16* dst = p.o + (qrow * p.n_heads + h) * D + lane * V;
-        if constexpr (V == 4) {
-            __nv_bfloat162 a = __floats2bfloat162_rn(acc[0], acc[1]);
-            __nv_bfloat162 b = __floats2bfloat162_rn(acc[2], acc[3]);
-            uint2 o2;
-            o2.x = *reinterpret_cast<uint32_t*>(&a);
-            o2.y = *reinterpret_cast<uint32_t*>(&b);
-            *reinterpret_cast<uint2*>(dst) = o2;
-        } else {
-            *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(acc[0], acc[1]);
+        for (int h = h_begin; h < h_end; ++h) {
+            float acc[V];
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[i] = 0.f;
+            const float* src0 = p.o_partial + ((int64_t)row * p.n_heads + h) * D + lane * V;
+            const float* lse_h = p.lse_partial + (int64_t)h * p.partial_rows + row;
+            const float L = merge_one<D, NP>(p, g, part, slot, src0, lse_h, acc);
+            __nv_bfloat16* dst = p.o + (qrow * p.n_heads + h) * D + lane * V;
+            if constexpr (V == 4) {
+                __nv_bfloat162 a = __floats2bfloat162_rn(acc[0], acc[1]);
+                __nv_bfloat162 b = __floats2bfloat162_rn(acc[2], acc[3]);
+                uint2 o2;
+                o2.x = *reinterpret_cast<uint32_t*>(&a);
+                o2.y = *reinterpret_cast<uint32_t*>(&b);
+                *reinterpret_cast<uint2*>(dst) = o2;
+            } else {
+                *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(acc[0], acc[1]);
+            }
+            if (lane == 0) p.lse[(int64_t)h * p.total_q + qrow] = L;
         }
-        if (lane == 0) p.lse[(int64_t)h * p.total_q + qrow] = L;
     }
 }
 
@@ -130,7 +156,7 @@ __global__ void __launch_bounds__(kMergeThreads, 8) zl_merge_kernel(const MergeP
 
 cudaError_t launch_merge(int head_dim, const MergeParams& p, int max_parts, int n_sms, cudaStream_t stream) {
     if (p.n_groups == 0) return cudaSuccess;
-    const int grid = n_sms * 8;  // 8 resident blocks of 256 threads per SM
+    const int grid = n_sms * 8;
     const int np = max_parts <= 4 ? 4 : (max_parts <= 8 ? 8 : 0);
     if (head_dim == 128) {
         if (np == 4) zl_merge_kernel<128, 4><<<grid, kMergeThreads, 0, stream>>>(p);
