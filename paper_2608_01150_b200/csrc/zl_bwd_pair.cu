@@ -65,7 +65,8 @@ struct PairSmem {
     alignas(1024) uint8_t aug_d[2048];              // [pieces of -D | zeros]
     alignas(1024) uint8_t ones[2][2048];            // [ones in elements 0..2][zeros]
     alignas(8) uint64_t kv_full, kv_empty, kx_empty;
-    uint64_t qr_full, qr_empty, qc_full, qc_empty, do_full, do_empty;
+    uint64_t qr_full, qr_empty, qc_full, qc_empty;
+    uint64_t dor_full, dor_empty, doc_full, doc_empty;  // dO rows + D pieces (B of dP^T) and dO columns (B of dV) have different lifetimes
     uint64_t s_full, dp_full, p_full, dst_full, ds_full, ds_free, dq_full, acc_full;
     uint64_t dq_empty[2];  // dQ tile g drained from TMEM: barrier g & 1 (two waiters, one of which may be two tiles behind)
     uint64_t s_read;      // every P/dS warp of both CTAs has read its S^T columns
@@ -147,8 +148,10 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mbar_init(&sm.qr_empty, 1);
         mbar_init(&sm.qc_full, 1);
         mbar_init(&sm.qc_empty, 1);
-        mbar_init(&sm.do_full, 1);
-        mbar_init(&sm.do_empty, 1);
+        mbar_init(&sm.dor_full, 1);
+        mbar_init(&sm.dor_empty, 1);
+        mbar_init(&sm.doc_full, 1);
+        mbar_init(&sm.doc_empty, 1);
         mbar_init(&sm.s_full, 1);
         mbar_init(&sm.dp_full, 1);
         mbar_init(&sm.p_full, 16);    // one arrival per P/dS warp of both CTAs
@@ -205,7 +208,8 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // producer arms for the pair.
             const uint32_t kv_full_l = map_to_cta(smem_u32(&sm.kv_full), 0);
             const uint32_t qr_full_l = map_to_cta(smem_u32(&sm.qr_full), 0);
-            const uint32_t do_full_l = map_to_cta(smem_u32(&sm.do_full), 0);
+            const uint32_t dor_full_l = map_to_cta(smem_u32(&sm.dor_full), 0);
+            const uint32_t doc_full_l = map_to_cta(smem_u32(&sm.doc_full), 0);
             uint32_t item_cnt = 0, it_cnt = 0;
             for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
                 const WorkItem wi = p.items[it];
@@ -230,13 +234,14 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         for (int b = 0; b < 2; ++b)
                             tma_load_3d_pair(sm.q_r[b], &tm_q64, qr_full_l, b * 64, wi.head, q0 + 64 * (int)rank);
                         tma_load_2d_pair(sm.aug_s, &tm_aug, qr_full_l, 0, aug_row);
-                        ZL_WAIT(&sm.do_empty, (it_cnt & 1) ^ 1, 3);
-                        if (rank == 0)
-                            mbar_arrive_expect_tx(&sm.do_full, 2 * (2 * Smem::kHalfBoxBytes + Smem::kBoxBytes + 1024));
+                        ZL_WAIT(&sm.dor_empty, (it_cnt & 1) ^ 1, 3);
+                        if (rank == 0) mbar_arrive_expect_tx(&sm.dor_full, 2 * (2 * Smem::kHalfBoxBytes + 1024));
                         for (int b = 0; b < 2; ++b)
-                            tma_load_3d_pair(sm.do_r[b], &tm_do64, do_full_l, b * 64, wi.head, q0 + 64 * (int)rank);
-                        tma_load_3d_pair(sm.do_c, &tm_do, do_full_l, 64 * (int)rank, wi.head, q0);
-                        tma_load_2d_pair(sm.aug_d, &tm_aug, do_full_l, 0, aug_row + 2);
+                            tma_load_3d_pair(sm.do_r[b], &tm_do64, dor_full_l, b * 64, wi.head, q0 + 64 * (int)rank);
+                        tma_load_2d_pair(sm.aug_d, &tm_aug, dor_full_l, 0, aug_row + 2);
+                        ZL_WAIT(&sm.doc_empty, (it_cnt & 1) ^ 1, 7);
+                        if (rank == 0) mbar_arrive_expect_tx(&sm.doc_full, 2 * Smem::kBoxBytes);
+                        tma_load_3d_pair(sm.do_c, &tm_do, doc_full_l, 64 * (int)rank, wi.head, q0);
                     }
                 }
             }
@@ -309,13 +314,14 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 if (mma_lane) mma_ss_pair(tmem + kColDP, dones, daug_d, idesc_s, true);
                 if (mma_lane) mma_commit_pair(&sm.dp_full);
+                if (mma_lane) mma_commit_pair(&sm.dor_empty);
             };
             auto issue_dv = [&](bool acc) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // dV += P^T dO, K = 128 query rows
                     if (mma_lane) mma_ts_pair(tmem + kColDV, tmem + kColS + ks * 8, ddoc_mn + ks * (2048 >> 4), idesc_kv,
                                               acc || ks > 0);
-                if (mma_lane) mma_commit_pair(&sm.do_empty);
+                if (mma_lane) mma_commit_pair(&sm.doc_empty);
             };
             uint32_t item_cnt = 0, it_cnt = 0;
             uint32_t dq_waited = 0;  // dQ tiles known to be drained from TMEM in both CTAs
@@ -332,10 +338,11 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 while (dq_waited < it_cnt) { ZL_WAIT_WARP_CL(&sm.dq_empty[dq_waited & 1], (dq_waited >> 1) & 1, 14); ++dq_waited; }
                 tc_fence_after();
                 issue_s();
-                ZL_WAIT_WARP_CL(&sm.do_full, it_cnt & 1, 13);
+                ZL_WAIT_WARP_CL(&sm.dor_full, it_cnt & 1, 13);
                 tc_fence_after();
                 issue_dp();
                 ZL_WAIT_WARP_CL(&sm.p_full, it_cnt & 1, 15);
+                ZL_WAIT_WARP_CL(&sm.doc_full, it_cnt & 1, 28);
                 tc_fence_after();
                 issue_dv(false);
                 if (n_it > 1) {
@@ -355,10 +362,11 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (mma_lane) mma_commit_pair(&sm.qc_empty);
                     if (i + 1 < n_it) {
                         // dP^T of the next tile right behind it (it overwrites dS^T: ordered after dK on the tensor pipe)
-                        ZL_WAIT_WARP_CL(&sm.do_full, (it_cnt + 1) & 1, 19);
+                        ZL_WAIT_WARP_CL(&sm.dor_full, (it_cnt + 1) & 1, 19);
                         tc_fence_after();
                         issue_dp();
                         ZL_WAIT_WARP_CL(&sm.p_full, (it_cnt + 1) & 1, 21);
+                        ZL_WAIT_WARP_CL(&sm.doc_full, (it_cnt + 1) & 1, 29);
                         tc_fence_after();
                         issue_dv(true);
                         if (i + 2 < n_it) {
