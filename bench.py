@@ -600,6 +600,17 @@ def run_cp(args):
     dist.destroy_process_group()
 
 
+def run_profile(args):
+    """Hardware-profiler record (paper Section IV-B / V-B): the price table of the paper's catalog on this GPU, the
+    catalog cut it implies, and the additive model checked on the covering plans; one JSON line."""
+    import torch
+    from paper_2608_01150_b200 import profiler
+    torch.cuda.set_device(0)
+    rep = profiler.catalog_report(args.profile_heads, 128, steps=3)
+    rep = {"mode": "profile", **rep}
+    print(json.dumps(rep), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -612,6 +623,10 @@ def main():
     ap.add_argument("--fuse-local-chunks", action="store_true",
                     help="build the handle with ZL_BUILD_FUSE_LOCAL_CHUNKS: query ranges whose chunks are contiguous run "
                          "as one final task (no partials, nothing to merge); off by default")
+    ap.add_argument("--profile", action="store_true",
+                    help="print the hardware profiler's record (price table of the paper's catalog, catalog cut, additivity) "
+                         "instead of the benchmark line")
+    ap.add_argument("--profile-heads", type=int, default=12)
     ap.add_argument("--cp", action="store_true",
                     help="context-parallel mode: one video under N-way all-gather CP across the N ranks + images per rank, "
                          "through the executor (printed as its own JSON line, not the headline)")
@@ -623,6 +638,9 @@ def main():
 
     if args.ablation:
         run_ablation(args)
+        return
+    if args.profile:
+        run_profile(args)
         return
 
     if args.impl == "reference":

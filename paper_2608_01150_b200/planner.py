@@ -21,6 +21,8 @@ def catalog_cut(whole_prices: Sequence[float]) -> int:
         raise ValueError("a cut needs at least two buckets")
     if np.any(np.diff(w) < 0):
         raise ValueError("buckets must be ordered by nondecreasing price")
+    if not np.all(np.isfinite(w)) or np.any(w <= 0):
+        raise ValueError("prices must be positive and finite (the cut works on their logarithms)")
     x = np.log(w)
     x = x - x.mean()                       # the dispersion is shift-invariant; centring keeps the sums small
     s1, s2 = np.cumsum(x), np.cumsum(x * x)

@@ -28,6 +28,18 @@ from typing import Callable, Dict, List, Optional, Sequence, Tuple
 BUCKETS: Dict[str, int] = {"image_480p": 1560, "video_480p": 32760, "video_720p": 75600}
 DEGREES: Tuple[int, ...] = (1, 2, 4, 8)
 
+# The catalog of the paper's evaluation (Section V-A: 256p-1080p images, 480p-1080p videos of 5, 10 and 15
+# seconds): tokens per latent frame x latent frames.  A 1080p frame is 8,160 tokens and a 15-second clip has 61
+# latent frames, which gives the 497,760-token sequence of the paper's introduction; 10 s = 41 frames, 5 s = 21.
+FRAME_TOKENS = {"256p": 256, "480p": 1560, "720p": 3600, "1080p": 8160}
+LATENT_FRAMES = {"5s": 21, "10s": 41, "15s": 61}
+CATALOG: Dict[str, int] = {f"image_{r}": t for r, t in FRAME_TOKENS.items()}
+CATALOG.update({f"video_{r}_{d}": FRAME_TOKENS[r] * n for r in ("480p", "720p", "1080p") for d, n in LATENT_FRAMES.items()})
+CATALOG_DEGREES: Tuple[int, ...] = (1, 2, 4, 8, 16)
+# a (bucket, degree) pair is profiled when the rank's share is at most this many score pairs per head
+# (a whole 15-second 1080p video on one rank is 2.5e11 pairs: seconds per step, and no planner would place it so)
+MAX_PAIRS_PER_HEAD = 3.2e10
+
 
 @dataclass(frozen=True)
 class Segment:
@@ -117,17 +129,54 @@ def gpu_timer(n_heads: int, head_dim: int, steps: int = 5, warmup: int = 2) -> C
 
 
 def profile_prices(measure: Callable[[Sequence[Segment]], float], buckets: Dict[str, int] = BUCKETS,
-                   degrees: Sequence[int] = DEGREES) -> Tuple[Dict[str, float], float]:
+                   degrees: Sequence[int] = DEGREES, max_pairs: float = float("inf")) -> Tuple[Dict[str, float], float]:
     """Measures every bucket x degree alone.  The placement-independent step cost is the time of a step
-    over one 128-token sequence (five launches that do next to nothing); it is removed from every price."""
+    over one 128-token sequence (five launches that do next to nothing); it is removed from every price.
+    Pairs whose chunks would be shorter than one tile, or whose rank share exceeds `max_pairs` score pairs
+    per head, are not profiled."""
     step_cost = measure([Segment("floor", 128, 1)])
     prices = {}
     for name, tokens in buckets.items():
         for k in degrees:
-            if tokens // k < 128:
+            if tokens // k < 128 or (tokens / k) * tokens > max_pairs:
                 continue
-            prices[f"{name}@{k}"] = max(0.0, measure([Segment(name, tokens, k)]) - step_cost)
+            # a sequence that costs no more than the placement-independent floor gets the timer's resolution
+            # (1 us): prices enter the catalog cut through their logarithm
+            prices[f"{name}@{k}"] = max(1e-3, measure([Segment(name, tokens, k)]) - step_cost)
     return prices, step_cost
+
+
+def whole_prices(prices: Dict[str, float], buckets: Dict[str, int]) -> Dict[str, float]:
+    """Price of every bucket run as ONE sequence on one rank, the quantity the catalog cut (Eq. 3) orders the
+    buckets by: the degree-1 price where it was measured, else k times the price of the smallest profiled
+    degree k (the k chunks of a sequence cost the same on every rank, and together they are the sequence)."""
+    out = {}
+    for name in buckets:
+        ks = sorted(int(key.split("@")[1]) for key in prices if key.split("@")[0] == name)
+        if ks:
+            out[name] = ks[0] * prices[f"{name}@{ks[0]}"]
+    return out
+
+
+def covering_plans(prices: Dict[str, float], buckets: Dict[str, int], n_images: int = 50,
+                   image: str = "image_480p", duration: str = "5s") -> List[List[Segment]]:
+    """Mixed plans in the manner of Section V-B: every plan holds one 480p, one 720p and one 1080p video of
+    `duration` plus a fixed set of images, and the profiled degrees rotate over the resolutions so that every
+    (resolution, degree) pair that was profiled occurs; then the all-whole corner plans (images only; three
+    480p videos + images; three 720p videos + images)."""
+    videos = [f"video_{r}_{duration}" for r in ("480p", "720p", "1080p") if f"video_{r}_{duration}" in buckets]
+    img = [Segment(image, buckets[image], 1)] * n_images
+    degs = {v: sorted(int(k.split("@")[1]) for k in prices if k.split("@")[0] == v) for v in videos}
+    n = max(len(d) for d in degs.values())
+    plans = []
+    for r in range(n):
+        plan = [Segment(v, buckets[v], degs[v][(r + i) % len(degs[v])]) for i, v in enumerate(videos)]
+        plans.append(plan + img)
+    plans.append(list(img))
+    for v in videos[:2]:
+        if 1 in degs[v]:
+            plans.append([Segment(v, buckets[v], 1)] * 3 + img)
+    return plans
 
 
 def rotation_plans(buckets: Dict[str, int] = BUCKETS, degrees: Sequence[int] = DEGREES,
@@ -158,14 +207,39 @@ def check_additivity(measure, prices, step_cost, plans) -> Dict:
             "mae_ms": sum(abs(r["predicted_ms"] - r["measured_ms"]) for r in rows) / max(1, len(rows))}
 
 
+def catalog_report(n_heads: int, head_dim: int, steps: int = 3, n_images: int = 50, duration: str = "5s") -> Dict:
+    """Profiles the paper's catalog on cuda:0 and checks the additive model on the covering plans; also applies
+    the catalog cut (Eq. 3) to the whole-sequence prices.  Returns a JSON-ready dict."""
+    from . import planner
+    measure = gpu_timer(n_heads, head_dim, steps=steps, warmup=1)
+    prices, step_cost = profile_prices(measure, CATALOG, CATALOG_DEGREES, MAX_PAIRS_PER_HEAD)
+    whole = whole_prices(prices, CATALOG)
+    fillers, anchors = planner.split_catalog(whole)
+    plans = covering_plans(prices, CATALOG, n_images=n_images, duration=duration)
+    return {"n_heads": n_heads, "head_dim": head_dim, "step_cost_ms": step_cost, "prices_ms": prices,
+            "whole_prices_ms": whole, "catalog_cut": {"fillers": fillers, "anchors": anchors},
+            "additivity": check_additivity(measure, prices, step_cost, plans)}
+
+
 def main(argv: Optional[Sequence[str]] = None) -> int:
     ap = argparse.ArgumentParser(description=__doc__.split("\n\n")[0])
     ap.add_argument("--heads", type=int, default=12)
     ap.add_argument("--head-dim", type=int, default=128)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--images", type=int, default=16)
+    ap.add_argument("--catalog", action="store_true",
+                    help="profile the paper's catalog (256p-1080p images, 480p-1080p videos of 5/10/15 s, degrees 1-16) "
+                         "and check the additive model on the covering plans of its Section V-B")
     ap.add_argument("--out", default="")
     args = ap.parse_args(argv)
+    if args.catalog:
+        report = catalog_report(args.heads, args.head_dim, steps=min(args.steps, 3), n_images=max(args.images, 50))
+        text = json.dumps(report, indent=1)
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text)
+        print(text)
+        return 0
     measure = gpu_timer(args.heads, args.head_dim, steps=args.steps)
     prices, step_cost = profile_prices(measure)
     report = {"n_heads": args.heads, "head_dim": args.head_dim, "step_cost_ms": step_cost, "prices_ms": prices,
