@@ -39,6 +39,9 @@ CATALOG_DEGREES: Tuple[int, ...] = (1, 2, 4, 8, 16)
 # a (bucket, degree) pair is profiled when the rank's share is at most this many score pairs per head
 # (a whole 15-second 1080p video on one rank is 2.5e11 pairs: seconds per step, and no planner would place it so)
 MAX_PAIRS_PER_HEAD = 3.2e10
+# small buckets are priced from a batch with at least this many query rows (a few waves of 256-row work items on
+# 148 SMs at 12 heads)
+FILL_ROWS = 16384
 
 
 @dataclass(frozen=True)
@@ -129,20 +132,25 @@ def gpu_timer(n_heads: int, head_dim: int, steps: int = 5, warmup: int = 2) -> C
 
 
 def profile_prices(measure: Callable[[Sequence[Segment]], float], buckets: Dict[str, int] = BUCKETS,
-                   degrees: Sequence[int] = DEGREES, max_pairs: float = float("inf")) -> Tuple[Dict[str, float], float]:
-    """Measures every bucket x degree alone.  The placement-independent step cost is the time of a step
-    over one 128-token sequence (five launches that do next to nothing); it is removed from every price.
-    Pairs whose chunks would be shorter than one tile, or whose rank share exceeds `max_pairs` score pairs
-    per head, are not profiled."""
+                   degrees: Sequence[int] = DEGREES, max_pairs: float = float("inf"),
+                   fill_rows: int = 0) -> Tuple[Dict[str, float], float]:
+    """Measures every bucket x degree.  The placement-independent step cost is the time of a step over one
+    128-token sequence (five launches that do next to nothing); it is removed from every price.  Pairs whose
+    chunks would be shorter than one tile, or whose rank share exceeds `max_pairs` score pairs per head, are
+    not profiled.  A bucket too small to fill the GPU on its own is measured as a batch of identical sequences
+    with at least `fill_rows` query rows in total and priced per sequence: one image alone leaves most SMs
+    idle, which is not what it costs inside a batch (the paper's measurements include packing)."""
     step_cost = measure([Segment("floor", 128, 1)])
     prices = {}
     for name, tokens in buckets.items():
         for k in degrees:
             if tokens // k < 128 or (tokens / k) * tokens > max_pairs:
                 continue
+            seg = Segment(name, tokens, k)
+            n = max(1, -(-fill_rows // seg.chunk())) if fill_rows else 1
             # a sequence that costs no more than the placement-independent floor gets the timer's resolution
             # (1 us): prices enter the catalog cut through their logarithm
-            prices[f"{name}@{k}"] = max(1e-3, measure([Segment(name, tokens, k)]) - step_cost)
+            prices[f"{name}@{k}"] = max(1e-3, (measure([seg] * n) - step_cost) / n)
     return prices, step_cost
 
 
@@ -212,7 +220,7 @@ def catalog_report(n_heads: int, head_dim: int, steps: int = 3, n_images: int = 
     the catalog cut (Eq. 3) to the whole-sequence prices.  Returns a JSON-ready dict."""
     from . import planner
     measure = gpu_timer(n_heads, head_dim, steps=steps, warmup=1)
-    prices, step_cost = profile_prices(measure, CATALOG, CATALOG_DEGREES, MAX_PAIRS_PER_HEAD)
+    prices, step_cost = profile_prices(measure, CATALOG, CATALOG_DEGREES, MAX_PAIRS_PER_HEAD, fill_rows=FILL_ROWS)
     whole = whole_prices(prices, CATALOG)
     fillers, anchors = planner.split_catalog(whole)
     plans = covering_plans(prices, CATALOG, n_images=n_images, duration=duration)

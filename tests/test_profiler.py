@@ -69,18 +69,18 @@ def test_catalog_covers_the_paper_buckets_and_plans():
 
 @pytest.mark.gpu
 def test_profile_medium_buckets_on_gpu():
-    """Sequences of 2-8 K tokens at 4 heads, d = 128: prices measured alone predict mixed plans within 10 %
-    (launch and tail effects of tiny sequences are gone at this size), and the measured whole-sequence prices
+    """Images of 1.5-4 K tokens and videos of 16-32 K tokens at 12 heads, d = 128: prices (small buckets priced
+    from a batch that fills the GPU) predict mixed plans within 10 %, and the measured whole-sequence prices
     drive the catalog cut."""
     from paper_2608_01150_b200 import planner
     buckets = {"image_a": 1560, "image_b": 3600, "video_a": 16384, "video_b": 32760}
-    measure = P.gpu_timer(4, 128, steps=5, warmup=2)
-    prices, step_cost = P.profile_prices(measure, buckets, (1, 2, 4))
+    measure = P.gpu_timer(12, 128, steps=5, warmup=2)
+    prices, step_cost = P.profile_prices(measure, buckets, (1, 2, 4), fill_rows=P.FILL_ROWS)
     assert step_cost > 0 and all(np.isfinite(v) and v > 0 for v in prices.values()) and len(prices) == 12
     # prices grow with the rank's share of the work: L^2 / k
     for b in buckets:
         assert prices[f"{b}@1"] > prices[f"{b}@2"] > prices[f"{b}@4"]
-    plans = P.rotation_plans({k: v for k, v in buckets.items() if k != "image_b"}, (1, 2, 4), n_images=8)
+    plans = P.rotation_plans({k: v for k, v in buckets.items() if k != "image_b"}, (1, 2, 4), n_images=16)
     rep = P.check_additivity(measure, prices, step_cost, plans)
     print("additivity:", [(r["plan"][:2], round(r["error_pct"], 2)) for r in rep["plans"]], rep["mape_pct"])
     assert rep["mape_pct"] <= 10.0, rep
