@@ -79,21 +79,46 @@ struct PairSmem {
 
 static_assert(sizeof(PairSmem) <= 227 * 1024, "shared memory of the pair kernel");
 
-__device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_flag, int where) {
+// Out of line, like the slow halves of the waits: the kernel has some sixty wait sites and its loops should stay in
+// the instruction cache.
+__device__ __noinline__ void report(int32_t* status, volatile int32_t* abort_flag, int where) {
     *abort_flag = 1;
     if (atomicCAS(status, 0, (int)ZL_ERR_TIMEOUT) == 0) status[1] = where;
 }
 
+// Bounded waits: the first try is inline, the timed loop out of line -- the kernel has some sixty wait sites and its
+// loops should stay in the instruction cache.  The loop gives up when the limit has passed or another role of the CTA
+// has given up; the acquire has cluster scope, which barriers the partner CTA arrives on need.
+__device__ __noinline__ bool pair_wait_slow(uint64_t* bar, uint32_t parity, const volatile int32_t* abort_flag) {
+    const uint64_t t0 = globaltimer();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((++spins & 0xFF) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer() - t0 > kWaitLimitNs) return false;
+        }
+    }
+}
+__device__ __forceinline__ bool pair_wait(uint64_t* bar, uint32_t parity, const volatile int32_t* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return pair_wait_slow(bar, parity, abort_flag);
+}
+__device__ __forceinline__ bool pair_wait_cluster(uint64_t* bar, uint32_t parity, const volatile int32_t* abort_flag) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    return pair_wait_slow(bar, parity, abort_flag);
+}
+
 #define ZL_WAIT(bar, parity, site)                                        \
     do {                                                                  \
-        if (!mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag)) { \
+        if (!pair_wait((bar), (parity), &sm.abort_flag)) {               \
             report(p.status, &sm.abort_flag, 3000 + (site));              \
             goto teardown;                                                \
         }                                                                 \
     } while (0)
 #define ZL_WAIT_WARP(bar, parity, site)                                              \
     do {                                                                             \
-        const bool ok_ = mbar_wait((bar), (parity), kWaitLimitNs, &sm.abort_flag); \
+        const bool ok_ = pair_wait((bar), (parity), &sm.abort_flag);                 \
         if (!__all_sync(0xffffffffu, ok_)) {                                         \
             report(p.status, &sm.abort_flag, 3000 + (site));                         \
             goto teardown;                                                           \
@@ -102,7 +127,7 @@ __device__ __forceinline__ void report(int32_t* status, volatile int32_t* abort_
 // the same for barriers the partner CTA arrives on
 #define ZL_WAIT_WARP_CL(bar, parity, site)                                                    \
     do {                                                                                      \
-        const bool ok_ = mbar_wait_cluster((bar), (parity), kWaitLimitNs, &sm.abort_flag); \
+        const bool ok_ = pair_wait_cluster((bar), (parity), &sm.abort_flag);                  \
         if (!__all_sync(0xffffffffu, ok_)) {                                                  \
             report(p.status, &sm.abort_flag, 3000 + (site));                                  \
             goto teardown;                                                                    \
@@ -201,7 +226,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const uint32_t tmem = sm.tmem_base;
 
     if (warp < 4) {
-        reg_dec<104>();
+        // (no register reallocation: every role fits the 128 registers the launch bounds give)
         if (warp == 0 && lane == 0) {
             // -------------------------------------------------------------- TMA producer: K, V, Q rows, dO
             // Transaction bytes of both CTAs are counted on the leader's barrier, which the leader's
@@ -323,60 +348,51 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                               acc || ks > 0);
                 if (mma_lane) mma_commit_pair(&sm.doc_empty);
             };
-            uint32_t item_cnt = 0, it_cnt = 0;
+            uint32_t item_cnt = 0, it_base = 0;  // it_base: query tiles of earlier items
             uint32_t dq_waited = 0;  // dQ tiles known to be drained from TMEM in both CTAs
             for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
                 const int n_it = count_q_tiles(p, g);
                 ZL_WAIT_WARP_CL(&sm.kv_full, item_cnt & 1, 11);
-                // prologue: S, dP, dV of the item's first query tile and S of the second.
-                // Steady-state order of this warp's MMAs: dK(i) dP(i+1) dV(i+1) S(i+2); dQ(i) comes from the second
-                // issuer.  S^T(x) overwrites the columns of dQ(x-2) (dQ(x-1) is only issued once S^T(x) has been
-                // read); the first S^T of an item follows the previous item's last dQ.
-                ZL_WAIT_WARP_CL(&sm.qr_full, it_cnt & 1, 12);
-                while (dq_waited < it_cnt) { ZL_WAIT_WARP_CL(&sm.dq_empty[dq_waited & 1], (dq_waited >> 1) & 1, 14); ++dq_waited; }
-                tc_fence_after();
-                issue_s();
-                ZL_WAIT_WARP_CL(&sm.dor_full, it_cnt & 1, 13);
-                tc_fence_after();
-                issue_dp();
-                ZL_WAIT_WARP_CL(&sm.p_full, it_cnt & 1, 15);
-                ZL_WAIT_WARP_CL(&sm.doc_full, it_cnt & 1, 28);
-                tc_fence_after();
-                issue_dv(false);
-                if (n_it > 1) {
-                    ZL_WAIT_WARP_CL(&sm.qr_full, (it_cnt + 1) & 1, 16);
-                    tc_fence_after();
-                    issue_s();  // overwrites P^T: ordered after dV on the tensor pipe
-                }
-                for (int i = 0; i < n_it; ++i, ++it_cnt) {
-                    // dK needs dS^T in TMEM only
-                    ZL_WAIT_WARP_CL(&sm.dst_full, it_cnt & 1, 17);
-                    ZL_WAIT_WARP_CL(&sm.qc_full, it_cnt & 1, 18);
-                    tc_fence_after();
+                // Order of this warp's MMAs: dK(i) dP(i+1) dV(i+1) S(i+2); dQ(i) comes from the second issuer.  The
+                // two steps before the item's first tile (i = -2, -1) are the prologue: S(0), then dP(0) dV(0) S(1).
+                // S^T(x) overwrites the columns of dQ(x-2) (dQ(x-1) is only issued once S^T(x) has been read); the
+                // first S^T of an item follows the previous item's last dQ.
+                for (int i = -2; i < n_it; ++i) {
+                    if (i >= 0) {
+                        // dK needs dS^T in TMEM only
+                        const uint32_t c = it_base + i;
+                        ZL_WAIT_WARP_CL(&sm.dst_full, c & 1, 17);
+                        ZL_WAIT_WARP_CL(&sm.qc_full, c & 1, 18);
+                        tc_fence_after();
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)  // dK += dS^T Q, K = 128 query rows, dS^T from TMEM
-                        if (mma_lane) mma_ts_pair(tmem + kColDK, tmem + kColDS + ks * 8, dqc_mn + ks * (2048 >> 4), idesc_kv,
-                                                  i > 0 || ks > 0);
-                    if (mma_lane) mma_commit_pair(&sm.qc_empty);
-                    if (i + 1 < n_it) {
+                        for (int ks = 0; ks < 8; ++ks)  // dK += dS^T Q, K = 128 query rows, dS^T from TMEM
+                            if (mma_lane) mma_ts_pair(tmem + kColDK, tmem + kColDS + ks * 8, dqc_mn + ks * (2048 >> 4), idesc_kv,
+                                                      i > 0 || ks > 0);
+                        if (mma_lane) mma_commit_pair(&sm.qc_empty);
+                    }
+                    if (i + 1 >= 0 && i + 1 < n_it) {
                         // dP^T of the next tile right behind it (it overwrites dS^T: ordered after dK on the tensor pipe)
-                        ZL_WAIT_WARP_CL(&sm.dor_full, (it_cnt + 1) & 1, 19);
+                        const uint32_t c = it_base + i + 1;
+                        ZL_WAIT_WARP_CL(&sm.dor_full, c & 1, 19);
                         tc_fence_after();
                         issue_dp();
-                        ZL_WAIT_WARP_CL(&sm.p_full, (it_cnt + 1) & 1, 21);
-                        ZL_WAIT_WARP_CL(&sm.doc_full, (it_cnt + 1) & 1, 29);
+                        ZL_WAIT_WARP_CL(&sm.p_full, c & 1, 21);
+                        ZL_WAIT_WARP_CL(&sm.doc_full, c & 1, 29);
                         tc_fence_after();
-                        issue_dv(true);
-                        if (i + 2 < n_it) {
-                            ZL_WAIT_WARP_CL(&sm.qr_full, (it_cnt + 2) & 1, 22);
-                            while (dq_waited < it_cnt + 1) { ZL_WAIT_WARP_CL(&sm.dq_empty[dq_waited & 1], (dq_waited >> 1) & 1, 25); ++dq_waited; }
-                            tc_fence_after();
-                            issue_s();
-                        }
+                        issue_dv(i + 1 > 0);
+                    }
+                    if (i + 2 < n_it) {
+                        const uint32_t c = it_base + i + 2;
+                        const uint32_t drained = it_base + (i + 1 > 0 ? i + 1 : 0);  // dQ tiles that must have left TMEM
+                        ZL_WAIT_WARP_CL(&sm.qr_full, c & 1, 22);
+                        while (dq_waited < drained) { ZL_WAIT_WARP_CL(&sm.dq_empty[dq_waited & 1], (dq_waited >> 1) & 1, 25); ++dq_waited; }
+                        tc_fence_after();
+                        issue_s();  // overwrites P^T: ordered after dV on the tensor pipe
                     }
                 }
+                it_base += n_it;
                 if (mma_lane) mma_commit_pair(&sm.acc_full);
                 if (mma_lane) mma_commit_pair(&sm.kv_empty);
             }
@@ -412,7 +428,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
     } else if (warp < 12) {
         // ------------------------------------------------------------------ P / dS warpgroups
-        reg_inc<128>();
+
         const int wg = (warp - 4) >> 2;            // 0: query columns 0-63, 1: columns 64-127
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;       // key row within this CTA's tile
@@ -435,12 +451,10 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const KvGroup g = p.kv_groups[wi.unit];
             const int rows_here = min(kTileKV, wi.rows - kTileKV * (int)rank);  // key rows of this CTA's tile (may be <= 0)
             const bool row_ok = row < rows_here;
-            for (int ti = 0; ti < g.n_tasks; ++ti) {
-                const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
-                const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
-                for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
-                    const int q_valid = min(kTileQ, t.q_len - qt * kTileQ);
-                    const bool tile_full = (rows_here == kTileKV) && (q_valid == kTileQ);  // warp-uniform
+            const float row_bias = row_ok ? 0.f : -INFINITY;
+            const int n_it = count_q_tiles(p, g);
+            {
+                for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 31);
                     tc_fence_after();
                     uint32_t pk[32];  // P^T of this thread's row, bf16 pairs
@@ -457,27 +471,15 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             mbar_arrive_cluster(s_read_l);
                             if (wg == 0) mbar_arrive(&sm.sp_read[quarter]);
                         }
-                        if (tile_full) {
+                        // S^T already has -LSE/scale folded in; query columns past the end of the task carry -1e30
+                        // there (preprocess kernel) and key rows past the end of the item get -inf here, so their
+                        // P is exactly zero without a second code path
 #pragma unroll
-                            for (int c = 0; c < 2; ++c)
+                        for (int c = 0; c < 2; ++c)
 #pragma unroll
-                                for (int i = 0; i < 32; i += 2)  // S^T already has -LSE/scale folded in
-                                    pk[c * 16 + i / 2] = pack_bf16(ex2(__uint_as_float(sr[c][i]) * sl2),
-                                                                   ex2(__uint_as_float(sr[c][i + 1]) * sl2));
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 2; ++c) {
-#pragma unroll
-                                for (int i = 0; i < 32; i += 2) {
-                                    const int col = col0 + c * 32 + i;
-                                    float p0 = ex2(__uint_as_float(sr[c][i]) * sl2);
-                                    float p1 = ex2(__uint_as_float(sr[c][i + 1]) * sl2);
-                                    p0 = (row_ok && col < q_valid) ? p0 : 0.f;  // select, never multiply
-                                    p1 = (row_ok && col + 1 < q_valid) ? p1 : 0.f;
-                                    pk[c * 16 + i / 2] = pack_bf16(p0, p1);
-                                }
-                            }
-                        }
+                            for (int i = 0; i < 32; i += 2)
+                                pk[c * 16 + i / 2] = pack_bf16(ex2(fmaf(__uint_as_float(sr[c][i]), sl2, row_bias)),
+                                                               ex2(fmaf(__uint_as_float(sr[c][i + 1]), sl2, row_bias)));
                         if (wg == 1) {
                             ZL_WAIT_WARP(&sm.sp_read[quarter], it_cnt & 1, 36);
                             tc_fence_after();
@@ -504,24 +506,14 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             if (lane == 0) mbar_arrive(&sm.dp_read[quarter]);
                         }
                         uint32_t dd[32];
+                        // dS^T = P^T o (dP^T - D) in packed bf16 arithmetic; where P is zero by masking, dP^T - D is
+                        // finite (rows of other sequences or the zero fill of the loads), so the product is zero
 #pragma unroll
-                        for (int c = 0; c < 2; ++c) {
-                            if (tile_full) {
+                        for (int c = 0; c < 2; ++c)
 #pragma unroll
-                                for (int i = 0; i < 32; i += 2)  // dS^T = P^T o (dP^T - D) in packed bf16 arithmetic
-                                    dd[c * 16 + i / 2] = mul_bf16x2(pk[c * 16 + i / 2],
-                                                                    pack_bf16(__uint_as_float(dr[c][i]), __uint_as_float(dr[c][i + 1])));
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < 32; i += 2) {
-                                    const int col = col0 + c * 32 + i;
-                                    float d0 = __uint_as_float(dr[c][i]), d1 = __uint_as_float(dr[c][i + 1]);
-                                    d0 = (row_ok && col < q_valid) ? d0 : 0.f;  // P is already zero there; keep 0 * garbage out
-                                    d1 = (row_ok && col + 1 < q_valid) ? d1 : 0.f;
-                                    dd[c * 16 + i / 2] = mul_bf16x2(pk[c * 16 + i / 2], pack_bf16(d0, d1));
-                                }
-                            }
-                        }
+                            for (int i = 0; i < 32; i += 2)
+                                dd[c * 16 + i / 2] = mul_bf16x2(pk[c * 16 + i / 2],
+                                                                pack_bf16(__uint_as_float(dr[c][i]), __uint_as_float(dr[c][i + 1])));
                         // A operand of dK first (dS^T as bf16 pairs in TMEM): the dK MMAs start while the rows for
                         // the dQ operand are still being stored and sent
                         if (wg == 1) {
@@ -582,7 +574,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // ------------------------------------------------------------------ dQ warpgroup
         // The CTA's dQ tile (its 64 query rows x 128 columns) sits in TMEM as 128 lanes x 64 columns: lanes
         // 0-63 hold columns 0-63 of rows 0-63, lanes 64-127 columns 64-127.  Warp w drains lanes 32w..32w+31.
-        reg_inc<152>();
+
         const int quarter = warp & 3;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const bool leader = (lane == 0);
