@@ -136,6 +136,7 @@ __device__ __forceinline__ bool pair_wait_cluster(uint64_t* bar, uint32_t parity
 
 __device__ __forceinline__ int count_q_tiles(const BwdParams& p, const KvGroup& g) {
     int n = 0;
+    #pragma unroll 1
     for (int ti = 0; ti < g.n_tasks; ++ti)
         n += (p.tasks[p.kv_group_tasks[g.task_begin + ti]].q_len + kTileQ - 1) / kTileQ;
     return n;
@@ -236,6 +237,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t dor_full_l = map_to_cta(smem_u32(&sm.dor_full), 0);
             const uint32_t doc_full_l = map_to_cta(smem_u32(&sm.doc_full), 0);
             uint32_t item_cnt = 0, it_cnt = 0;
+            #pragma unroll 1
             for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
@@ -248,9 +250,11 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     tma_load_3d_pair(sm.v + b * Smem::kBoxBytes, &tm_v, kv_full_l, b * 64, wi.head, key0 + 128 * (int)rank);
                     tma_load_3d_pair(sm.kx[b], &tm_k, kv_full_l, 64 * (int)rank, wi.head, key0 + 128 * b);
                 }
+                #pragma unroll 1
                 for (int ti = 0; ti < g.n_tasks; ++ti) {
                     const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                     const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
+                    #pragma unroll 1
                     for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
                         const int q0 = t.q_off + qt * kTileQ;
                         const int aug_row = (wi.head * (p.q_pad_total / kTileQ) + t.q_slot / kTileQ + qt) * 4 + (int)rank;
@@ -276,12 +280,15 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // from delaying the other loads.
             const uint32_t qc_full_l = map_to_cta(smem_u32(&sm.qc_full), 0);
             uint32_t it_cnt = 0;
+            #pragma unroll 1
             for (int it = cluster_id; it < p.n_items; it += n_clusters) {
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
+                #pragma unroll 1
                 for (int ti = 0; ti < g.n_tasks; ++ti) {
                     const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                     const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
+                    #pragma unroll 1
                     for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
                         ZL_WAIT(&sm.qc_empty, (it_cnt & 1) ^ 1, 4);
                         if (rank == 0) mbar_arrive_expect_tx(&sm.qc_full, 2 * Smem::kBoxBytes);
@@ -295,9 +302,11 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // have landed here, tell the leader.
             const uint32_t ds_full_l = map_to_cta(smem_u32(&sm.ds_full), 0);
             uint32_t it_cnt = 0;
+            #pragma unroll 1
             for (int it = cluster_id; it < p.n_items; it += n_clusters) {
                 const KvGroup g = p.kv_groups[p.items[it].unit];
                 const int n_it = count_q_tiles(p, g);
+                #pragma unroll 1
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     mbar_arrive_expect_tx(&sm.ds_land, Smem::kBoxBytes);
                     ZL_WAIT(&sm.ds_land, it_cnt & 1, 5);
@@ -350,6 +359,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             };
             uint32_t item_cnt = 0, it_base = 0;  // it_base: query tiles of earlier items
             uint32_t dq_waited = 0;  // dQ tiles known to be drained from TMEM in both CTAs
+            #pragma unroll 1
             for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
@@ -359,6 +369,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 // two steps before the item's first tile (i = -2, -1) are the prologue: S(0), then dP(0) dV(0) S(1).
                 // S^T(x) overwrites the columns of dQ(x-2) (dQ(x-1) is only issued once S^T(x) has been read); the
                 // first S^T of an item follows the previous item's last dQ.
+                #pragma unroll 1
                 for (int i = -2; i < n_it; ++i) {
                     if (i >= 0) {
                         // dK needs dS^T in TMEM only
@@ -406,10 +417,12 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint64_t dds_mn = make_desc_sw128(smem_u32(sm.ds[0]), Smem::kBoxBytes, 1024);
             const uint64_t dkx_mn = make_desc_sw128(smem_u32(sm.kx[0]), Smem::kBoxBytes, 1024);
             uint32_t item_cnt = 0, it_cnt = 0;
+            #pragma unroll 1
             for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
                 const KvGroup g = p.kv_groups[p.items[it].unit];
                 const int n_it = count_q_tiles(p, g);
                 ZL_WAIT_WARP_CL(&sm.kv_full, item_cnt & 1, 51);  // the K columns of this item are in place
+                #pragma unroll 1
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     ZL_WAIT_WARP_CL(&sm.ds_full, it_cnt & 1, 52);
                     if (i + 1 < n_it) ZL_WAIT_WARP_CL(&sm.s_read, (it_cnt + 1) & 1, 53);
@@ -446,6 +459,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t dst_full_l = map_to_cta(smem_u32(&sm.dst_full), 0);
         const float sl2 = p.scale_log2;
         uint32_t item_cnt = 0, it_cnt = 0;
+        #pragma unroll 1
         for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
             const WorkItem wi = p.items[it];
             const KvGroup g = p.kv_groups[wi.unit];
@@ -454,6 +468,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const float row_bias = row_ok ? 0.f : -INFINITY;
             const int n_it = count_q_tiles(p, g);
             {
+                #pragma unroll 1
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     ZL_WAIT_WARP(&sm.s_full, it_cnt & 1, 31);
                     tc_fence_after();
@@ -584,12 +599,15 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         uint8_t* buf = sm.dq_stage[quarter];
         const uint32_t row_addr = smem_u32(buf) + lane * 64;  // 64-byte rows, 64-byte swizzle
         uint32_t it_cnt = 0, chunk_cnt = 0;
+        #pragma unroll 1
         for (int it = cluster_id; it < p.n_items; it += n_clusters) {
             const WorkItem wi = p.items[it];
             const KvGroup g = p.kv_groups[wi.unit];
+            #pragma unroll 1
             for (int ti = 0; ti < g.n_tasks; ++ti) {
                 const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
                 const int n_q = (t.q_len + kTileQ - 1) / kTileQ;
+                #pragma unroll 1
                 for (int qt = 0; qt < n_q; ++qt, ++it_cnt) {
                     ZL_WAIT_WARP(&sm.dq_full, it_cnt & 1, 41);
                     tc_fence_after();
