@@ -303,7 +303,7 @@ zl_status zl_get_kernel_timing(zl_tasks* tasks, float* total_ms /* [ZL_K_COUNT] 
  * zl_last_device_status reports.  Nothing hangs and nothing faults. */
 zl_status zl_debug_set_fwd_order(zl_tasks* tasks, int32_t mode, void* stream);
 /* zl_set_bwd_kernel chooses the main kernel of zl_coalesced_attn_bwd for this handle: 0 = the library's
- * default, 1 = one CTA per 128-row key tile, 2 = pairs of CTAs (tcgen05 cta_group::2) that own two
+ * default (pairs at head_dim 128, one CTA otherwise), 1 = one CTA per 128-row key tile, 2 = pairs of CTAs (tcgen05 cta_group::2) that own two
  * neighbouring key tiles, share every B operand and sum dQ over 256 keys before it is reduced
  * (head_dim 128 only: ZL_ERR_UNSUPPORTED otherwise).  Results agree within the gradient tolerance; dK
  * and dV of the two kernels may differ in the last bit (different accumulation order). */

@@ -78,7 +78,7 @@ bool make_tmap(CUtensorMap* m, const void* base, int64_t rows, int n_heads, int 
 }
 
 constexpr int kMaxTimedLaunches = 1024;
-constexpr bool kDefaultBwdPair = false;  // which backward main kernel a handle uses unless zl_set_bwd_kernel chose one
+constexpr bool kDefaultBwdPair = true;   // which backward main kernel a handle uses unless zl_set_bwd_kernel chose one
 
 // Brackets one kernel launch with events when timing is enabled on the handle.
 struct LaunchTimer {
