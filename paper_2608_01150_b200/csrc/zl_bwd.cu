@@ -59,63 +59,90 @@ __device__ __forceinline__ void split3(float x, __nv_bfloat16 (&h)[3]) {
 template <int D>
 __global__ void __launch_bounds__(kPreThreads) zl_bwd_pre_kernel(const BwdParams p) {
     // One warp per (8 consecutive padded query rows, head): four lanes share a row, each reading a
-    // quarter of its O and dO (16-byte loads), so a warp keeps 4 KB (d=128) in flight and the two
-    // 16-byte halves of the eight rows land in the augmentation tile as two contiguous 128-byte stores.
+    // quarter of its O and dO (16-byte loads), and the two 16-byte halves of the eight rows land in the
+    // augmentation tile as two contiguous 128-byte stores.  A warp handles two such units per iteration and
+    // issues all loads of both (O, dO and LSE: 8 KB + 64 B at d=128) before the first use.
     constexpr int kPerLane = D / 4;  // bf16 elements of one row handled by one lane
+    constexpr int kVec = kPerLane / 8;
+    constexpr int kUnits = 2;
     const int lane = threadIdx.x & 31;
     const int sub = lane >> 2, quarter = lane & 3;
     const int64_t n_units = (int64_t)(p.q_pad_total / 8) * p.n_heads;
+    const int64_t stride = (int64_t)gridDim.x * (kPreThreads / 32);
     const float inv_scale = 1.f / p.scale;
-    for (int64_t u = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); u < n_units;
-         u += (int64_t)gridDim.x * (kPreThreads / 32)) {
-        const int row8 = (int)(u / p.n_heads);
-        const int h = (int)(u - (int64_t)row8 * p.n_heads);
-        const int slot_row = row8 * 8 + sub;
-        // slots are padded to 128 rows: the eight rows belong to one query group
-        const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, row8 * 8)];
-        if (h < g.head_begin || h >= g.head_begin + g.head_count) continue;  // warp-uniform: no task runs this head
-        const int r = slot_row - g.slot;
-        float xd = 0.f, xl = -1e30f;
-        const bool live = r < g.q_len;
-        float acc = 0.f;
-        if (live) {
-            const int64_t row = (int64_t)g.q_off + r;
-            const uint4* po = reinterpret_cast<const uint4*>(p.o + (row * p.n_heads + h) * D + quarter * kPerLane);
-            const uint4* pd = reinterpret_cast<const uint4*>(p.d_o + (row * p.n_heads + h) * D + quarter * kPerLane);
-            uint4 a[kPerLane / 8], b[kPerLane / 8];
+    for (int64_t u0 = (int64_t)blockIdx.x * (kPreThreads / 32) + (threadIdx.x >> 5); u0 < n_units; u0 += kUnits * stride) {
+        uint4 a[kUnits][kVec], b[kUnits][kVec];
+        float lse[kUnits];
+        bool live[kUnits], run[kUnits];
+        int slot_row[kUnits], head[kUnits];
 #pragma unroll
-            for (int i = 0; i < kPerLane / 8; ++i) { a[i] = __ldg(po + i); b[i] = __ldg(pd + i); }
+        for (int k = 0; k < kUnits; ++k) {
+            const int64_t u = u0 + k * stride;
+            run[k] = false;
+            live[k] = false;
+            lse[k] = 0.f;
+            slot_row[k] = 0;
+            head[k] = 0;
+            if (u >= n_units) continue;
+            const int row8 = (int)(u / p.n_heads);
+            const int h = (int)(u - (int64_t)row8 * p.n_heads);
+            // slots are padded to 128 rows: the eight rows belong to one query group
+            const QGroup g = p.q_groups[find_q_group(p.q_groups, p.n_q_groups, row8 * 8)];
+            if (h < g.head_begin || h >= g.head_begin + g.head_count) continue;  // warp-uniform: no task runs this head
+            run[k] = true;
+            head[k] = h;
+            slot_row[k] = row8 * 8 + sub;
+            const int r = slot_row[k] - g.slot;
+            live[k] = r < g.q_len;
+            if (live[k]) {
+                const int64_t row = (int64_t)g.q_off + r;
+                const uint4* po = reinterpret_cast<const uint4*>(p.o + (row * p.n_heads + h) * D + quarter * kPerLane);
+                const uint4* pd = reinterpret_cast<const uint4*>(p.d_o + (row * p.n_heads + h) * D + quarter * kPerLane);
 #pragma unroll
-            for (int i = 0; i < kPerLane / 8; ++i) {
-                const uint32_t aw[4] = {a[i].x, a[i].y, a[i].z, a[i].w}, bw[4] = {b[i].x, b[i].y, b[i].z, b[i].w};
-#pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[w]));
-                    const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[w]));
-                    acc = fmaf(fa.x, fb.x, acc);
-                    acc = fmaf(fa.y, fb.y, acc);
-                }
+                for (int i = 0; i < kVec; ++i) { a[k][i] = __ldg(po + i); b[k][i] = __ldg(pd + i); }
+                if (quarter == 0) lse[k] = __ldg(p.lse + (int64_t)h * p.total_q + row);
             }
         }
-        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-        if (live) {
-            xd = -acc;
-            const float l = p.lse[(int64_t)h * p.total_q + (int64_t)g.q_off + r];
-            if (l > -INFINITY && l < INFINITY) xl = -l * inv_scale;
-        }
-        // lane quarter 0 writes elements 0..7 of its row (-LSE/scale pieces), quarter 1 elements 8..15 (-D pieces)
-        if (quarter < 2) {
-            __nv_bfloat16 hp[3];
-            split3(quarter == 0 ? xl : xd, hp);
-            uint4 val;
-            val.x = (uint32_t)__bfloat16_as_ushort(hp[0]) | ((uint32_t)__bfloat16_as_ushort(hp[1]) << 16);
-            val.y = (uint32_t)__bfloat16_as_ushort(hp[2]);
-            val.z = 0u;
-            val.w = 0u;
-            const int tile = slot_row / kTileQ, tr = slot_row % kTileQ;
-            uint8_t* base = p.aug + ((int64_t)h * (p.q_pad_total / kTileQ) + tile) * 4096;
-            *reinterpret_cast<uint4*>(base + quarter * 2048 + (tr / 8) * 128 + (tr % 8) * 16) = val;
+#pragma unroll
+        for (int k = 0; k < kUnits; ++k) {
+            if (!run[k]) continue;  // warp-uniform
+            float acc = 0.f;
+            if (live[k]) {
+#pragma unroll
+                for (int i = 0; i < kVec; ++i) {
+                    const uint32_t aw[4] = {a[k][i].x, a[k][i].y, a[k][i].z, a[k][i].w};
+                    const uint32_t bw[4] = {b[k][i].x, b[k][i].y, b[k][i].z, b[k][i].w};
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[w]));
+                        const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[w]));
+                        acc = fmaf(fa.x, fb.x, acc);
+                        acc = fmaf(fa.y, fb.y, acc);
+                    }
+                }
+            }
+            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+            // rows past the end of the query range: -1e30 and 0, which makes their P and dS vanish
+            float xd = 0.f, xl = -1e30f;
+            if (live[k]) {
+                xd = -acc;
+                const float l = lse[k];
+                if (l > -INFINITY && l < INFINITY) xl = -l * inv_scale;
+            }
+            // lane quarter 0 writes elements 0..7 of its row (-LSE/scale pieces), quarter 1 elements 8..15 (-D pieces)
+            if (quarter < 2) {
+                __nv_bfloat16 hp[3];
+                split3(quarter == 0 ? xl : xd, hp);
+                uint4 val;
+                val.x = (uint32_t)__bfloat16_as_ushort(hp[0]) | ((uint32_t)__bfloat16_as_ushort(hp[1]) << 16);
+                val.y = (uint32_t)__bfloat16_as_ushort(hp[2]);
+                val.z = 0u;
+                val.w = 0u;
+                const int tile = slot_row[k] / kTileQ, tr = slot_row[k] % kTileQ;
+                uint8_t* base = p.aug + ((int64_t)head[k] * (p.q_pad_total / kTileQ) + tile) * 4096;
+                *reinterpret_cast<uint4*>(base + quarter * 2048 + (tr / 8) * 128 + (tr % 8) * 16) = val;
+            }
         }
     }
 }
