@@ -241,6 +241,53 @@ zl_status zl_coalesced_attn_bwd_packed(const zl_tasks* tasks, const void* qkv, c
                                        const void* d_o, float scale, void* dqkv,
                                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* Launch phases -- running the tasks of a handle in several launches, in the order their inputs arrive.
+ *
+ * Section IV-D runs the attention of a context-parallel rank under its collectives: the tasks whose K/V are
+ * already local start while the remaining K/V chunks are still on their way (all-gather, or one chunk per
+ * ring step), and in the backward the gradients of remote K/V chunks leave for their owners while the local
+ * ones are still being computed.  A phase is the unit of that overlap: the caller assigns every whole sequence
+ * and every shard a phase number, launches phase p when its inputs are there, and runs the merge once after
+ * the last forward phase.
+ *
+ * zl_set_fwd_phases: `whole_phase` [n_seqs] and `shard_phase` [n_shards] (host arrays; NULL = all zero) give
+ * the phase, 0 <= phase < n_phases <= ZL_MAX_PHASES, of every sequence / shard in the order they were passed
+ * to zl_build_tasks*.  The forward work list is regrouped by phase (longest-first inside each phase) and
+ * uploaded (the call synchronises `stream`).  A shard query range that the builder fused into one task
+ * (ZL_BUILD_FUSE_LOCAL_CHUNKS) runs in the latest phase of its shards.  zl_coalesced_attn_fwd still runs the
+ * whole list in one launch; zl_coalesced_attn_fwd_phase runs the tasks of one phase: arguments, outputs and
+ * errors as zl_coalesced_attn_fwd, plus ZL_ERR_INVALID_ARG for a phase the handle does not have.  K/V rows of
+ * tasks of later phases are not used, so they may still be in flight -- but a ragged last tile of a chunk is
+ * loaded whole, so the rows that follow a chunk must hold finite values at all times (zero the buffers once;
+ * a row that is half old and half new is still finite); O/LSE rows and partial slots of tasks of other phases
+ * are not written.  Phases may run in any order and on different streams; zl_lse_merge must
+ * follow all of them.  Results are bit-identical to the single launch.
+ *
+ * zl_set_bwd_phases: the same arrays for the backward.  The unit of the backward is the kv group (all tasks
+ * that share a key range: one work item finishes that range's dK and dV), which runs in the latest phase any of
+ * its tasks asks for.  zl_coalesced_attn_bwd_phase must be called for phase 0, 1, ..., n_phases-1 in this order
+ * on one stream with the same arguments: phase 0 first clears the dQ accumulator and forms D and -LSE/scale
+ * for all rows, every phase runs the main kernel over its kv groups, the last phase converts dQ.  After
+ * phase p has finished, the dK and dV rows of the kv groups of phases <= p are final (their reduce-scatter may
+ * start); dQ is final after the last phase.  dK and dV are bit-identical to zl_coalesced_attn_bwd, dQ up to the
+ * order of the fp32 reduce-adds.
+ *
+ * zl_phase_info reports the number of phases and the work items per phase (arrays of ZL_MAX_PHASES entries,
+ * any pointer may be NULL).  A handle starts with one phase per direction. */
+#define ZL_MAX_PHASES 64
+zl_status zl_set_fwd_phases(zl_tasks* tasks, const int32_t* whole_phase, const int32_t* shard_phase, int32_t n_phases,
+                            void* stream);
+zl_status zl_set_bwd_phases(zl_tasks* tasks, const int32_t* whole_phase, const int32_t* shard_phase, int32_t n_phases,
+                            void* stream);
+zl_status zl_coalesced_attn_fwd_phase(const zl_tasks* tasks, int32_t phase, const void* q, const void* k, const void* v,
+                                      float scale, void* o, float* lse, float* o_partial, float* lse_partial,
+                                      void* stream);
+zl_status zl_coalesced_attn_bwd_phase(const zl_tasks* tasks, int32_t phase, const void* q, const void* k, const void* v,
+                                      const void* o, const float* lse, const void* d_o, float scale,
+                                      void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes, void* stream);
+zl_status zl_phase_info(const zl_tasks* tasks, int32_t* n_fwd_phases, int32_t* n_bwd_phases,
+                        int32_t* fwd_items_per_phase /* [ZL_MAX_PHASES] */, int32_t* bwd_items_per_phase /* [ZL_MAX_PHASES] */);
+
 /* zl_coalesced_attn_bwd_noalloc -- the backward for callers that cannot allocate device memory.
  * (The paper has no counterpart; this is a convenience of the library.)
  *

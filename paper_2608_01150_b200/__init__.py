@@ -11,6 +11,7 @@ The names of :mod:`.binding` are resolved on first access, so that
 _BINDING_NAMES = ("ZlError", "TaskHandle", "ShardDesc", "WholeDesc", "HeadRange", "TasksInfo", "build_tasks",
                   "build_tasks_heads", "coalesced_attn_fwd", "lse_merge", "coalesced_attn_bwd",
                   "coalesced_attn_bwd_noalloc", "coalesced_attn_fwd_packed", "coalesced_attn_bwd_packed",
+                  "coalesced_attn_fwd_phase", "coalesced_attn_bwd_phase", "MAX_PHASES",
                   "NOALLOC_SCRATCH_BYTES", "BUILD_FUSE_LOCAL_CHUNKS", "launch_count", "library_path", "STATUS_NAMES")
 
 

@@ -86,6 +86,16 @@ def _load():
     lib.zl_coalesced_attn_bwd.restype = ctypes.c_int
     lib.zl_coalesced_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
+    for name in ("zl_set_fwd_phases", "zl_set_bwd_phases"):
+        getattr(lib, name).restype = ctypes.c_int
+        getattr(lib, name).argtypes = [vp, vp, vp, i32, vp]
+    lib.zl_coalesced_attn_fwd_phase.restype = ctypes.c_int
+    lib.zl_coalesced_attn_fwd_phase.argtypes = [vp, i32, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
+    lib.zl_coalesced_attn_bwd_phase.restype = ctypes.c_int
+    lib.zl_coalesced_attn_bwd_phase.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp,
+                                                ctypes.c_size_t, vp]
+    lib.zl_phase_info.restype = ctypes.c_int
+    lib.zl_phase_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.zl_coalesced_attn_bwd_noalloc.restype = ctypes.c_int
     lib.zl_coalesced_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.zl_last_device_status.restype = ctypes.c_int
@@ -189,6 +199,32 @@ class TaskHandle:
         """0 longest-first (default), 1 placement order, 2 shortest-first (measurement aid)."""
         _check(_lib.zl_debug_set_fwd_order(self._ptr, mode, _stream_ptr(stream)), "zl_debug_set_fwd_order")
 
+    @staticmethod
+    def _phase_array(values):
+        if values is None:
+            return None, None
+        arr = (ctypes.c_int32 * max(1, len(values)))(*[int(v) for v in values])
+        return arr, ctypes.cast(arr, ctypes.c_void_p)
+
+    def set_fwd_phases(self, whole_phase, shard_phase, n_phases: int, stream=None):
+        """zl_set_fwd_phases: one phase number per whole sequence / per shard (None = all zero)."""
+        a, ap = self._phase_array(whole_phase)
+        b, bp = self._phase_array(shard_phase)
+        _check(_lib.zl_set_fwd_phases(self._ptr, ap, bp, n_phases, _stream_ptr(stream)), "zl_set_fwd_phases")
+
+    def set_bwd_phases(self, whole_phase, shard_phase, n_phases: int, stream=None):
+        """zl_set_bwd_phases."""
+        a, ap = self._phase_array(whole_phase)
+        b, bp = self._phase_array(shard_phase)
+        _check(_lib.zl_set_bwd_phases(self._ptr, ap, bp, n_phases, _stream_ptr(stream)), "zl_set_bwd_phases")
+
+    def phase_info(self):
+        """zl_phase_info: (forward items per phase, backward items per phase)."""
+        nf, nb = ctypes.c_int32(0), ctypes.c_int32(0)
+        fi, bi = (ctypes.c_int32 * MAX_PHASES)(), (ctypes.c_int32 * MAX_PHASES)()
+        _check(_lib.zl_phase_info(self._ptr, ctypes.byref(nf), ctypes.byref(nb), fi, bi), "zl_phase_info")
+        return list(fi[:nf.value]), list(bi[:nb.value])
+
     def set_bwd_kernel(self, kernel: int):
         """0 library default, 1 one CTA per key tile, 2 CTA pairs (head_dim 128)."""
         _check(_lib.zl_set_bwd_kernel(self._ptr, kernel), "zl_set_bwd_kernel")
@@ -210,6 +246,7 @@ class TaskHandle:
 
 
 BUILD_FUSE_LOCAL_CHUNKS = 1
+MAX_PHASES = 64  # ZL_MAX_PHASES
 
 
 def build_tasks(cu_seqlens: Sequence[int], shards: Sequence[Sequence[int]], total_q: int, total_kv: int,
@@ -260,6 +297,25 @@ def coalesced_attn_fwd(tasks: TaskHandle, q, k, v, scale: float, o, lse, o_parti
     _check(_lib.zl_coalesced_attn_fwd(tasks.ptr, _ptr(q), _ptr(k), _ptr(v), ctypes.c_float(scale), _ptr(o),
                                       _ptr(lse), _ptr(o_partial), _ptr(lse_partial), _stream_ptr(stream)),
            "zl_coalesced_attn_fwd")
+
+
+def coalesced_attn_fwd_phase(tasks: TaskHandle, phase: int, q, k, v, scale: float, o, lse, o_partial=None,
+                             lse_partial=None, stream=None):
+    """zl_coalesced_attn_fwd_phase: the tasks of one launch phase."""
+    _check(_lib.zl_coalesced_attn_fwd_phase(tasks.ptr, phase, _ptr(q), _ptr(k), _ptr(v), ctypes.c_float(scale), _ptr(o),
+                                            _ptr(lse), _ptr(o_partial), _ptr(lse_partial), _stream_ptr(stream)),
+           "zl_coalesced_attn_fwd_phase")
+
+
+def coalesced_attn_bwd_phase(tasks: TaskHandle, phase: int, q, k, v, o, lse, d_o, scale: float, dq, dk, dv, workspace,
+                             workspace_bytes: Optional[int] = None, stream=None):
+    """zl_coalesced_attn_bwd_phase: phases 0 .. n-1 in order, same arguments."""
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(_lib.zl_coalesced_attn_bwd_phase(tasks.ptr, phase, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o),
+                                            ctypes.c_float(scale), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
+                                            ctypes.c_size_t(workspace_bytes), _stream_ptr(stream)),
+           "zl_coalesced_attn_bwd_phase")
 
 
 def lse_merge(tasks: TaskHandle, o_partial, lse_partial, o, lse, stream=None):

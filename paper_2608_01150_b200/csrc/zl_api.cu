@@ -340,10 +340,15 @@ void zl_free_tasks(zl_tasks* t) {
 
 namespace {
 // Forward over q, k, v given as token-major views with `in_stride` elements between rows.
-zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* v, int64_t in_stride, float scale,
-                   void* o, float* lse, float* o_partial, float* lse_partial, void* stream) {
+// `phase` < 0: the whole work list; otherwise the items of that launch phase only.
+zl_status fwd_impl(const zl_tasks* t, int32_t phase, const void* q, const void* k, const void* v, int64_t in_stride,
+                   float scale, void* o, float* lse, float* o_partial, float* lse_partial, void* stream) {
     const Schedule& s = t->sched;
-    if (s.fwd_items.empty()) return ZL_OK;
+    const int32_t n_phases = (int32_t)s.fwd_phase_begin.size() - 1;
+    if (phase >= n_phases) return ZL_ERR_INVALID_ARG;
+    const int32_t item_begin = phase < 0 ? 0 : s.fwd_phase_begin[phase];
+    const int32_t item_end = phase < 0 ? (int32_t)s.fwd_items.size() : s.fwd_phase_begin[phase + 1];
+    if (item_end == item_begin) return ZL_OK;
     if (t->device < 0) return ZL_ERR_CUDA;
     if (!on_handle_device(t)) return ZL_ERR_INVALID_ARG;
     if (!q || !k || !v || !o || !lse) return ZL_ERR_INVALID_ARG;
@@ -366,8 +371,8 @@ zl_status fwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
 
     FwdParams p{};
     p.tasks = t->d_tasks;
-    p.items = t->d_fwd_items;
-    p.n_items = (int32_t)s.fwd_items.size();
+    p.items = t->d_fwd_items + item_begin;
+    p.n_items = item_end - item_begin;
     p.n_heads = s.n_heads;
     p.total_q = s.total_q;
     p.partial_rows = (int32_t)s.partial_rows;
@@ -393,7 +398,15 @@ extern "C" {
 zl_status zl_coalesced_attn_fwd(const zl_tasks* t, const void* q, const void* k, const void* v, float scale,
                                 void* o, float* lse, float* o_partial, float* lse_partial, void* stream) {
     if (!t) return ZL_ERR_INVALID_ARG;
-    return fwd_impl(t, q, k, v, (int64_t)t->sched.n_heads * t->sched.head_dim, scale, o, lse, o_partial,
+    return fwd_impl(t, -1, q, k, v, (int64_t)t->sched.n_heads * t->sched.head_dim, scale, o, lse, o_partial,
+                    lse_partial, stream);
+}
+
+zl_status zl_coalesced_attn_fwd_phase(const zl_tasks* t, int32_t phase, const void* q, const void* k, const void* v,
+                                      float scale, void* o, float* lse, float* o_partial, float* lse_partial,
+                                      void* stream) {
+    if (!t || phase < 0) return ZL_ERR_INVALID_ARG;
+    return fwd_impl(t, phase, q, k, v, (int64_t)t->sched.n_heads * t->sched.head_dim, scale, o, lse, o_partial,
                     lse_partial, stream);
 }
 
@@ -405,7 +418,7 @@ zl_status zl_coalesced_attn_fwd_packed(const zl_tasks* t, const void* qkv, float
     if (!qkv) return s.fwd_items.empty() ? ZL_OK : ZL_ERR_INVALID_ARG;
     const int64_t hd = (int64_t)s.n_heads * s.head_dim;
     const __nv_bfloat16* base = static_cast<const __nv_bfloat16*>(qkv);
-    return fwd_impl(t, base, base + hd, base + 2 * hd, 3 * hd, scale, o, lse, o_partial, lse_partial, stream);
+    return fwd_impl(t, -1, base, base + hd, base + 2 * hd, 3 * hd, scale, o, lse, o_partial, lse_partial, stream);
 }
 
 zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* lse_partial, void* o, float* lse,
@@ -445,11 +458,16 @@ zl_status zl_lse_merge(const zl_tasks* t, const float* o_partial, const float* l
 namespace {
 // Backward over q, k, v views with `in_stride` elements between token rows and dq, dk, dv views
 // with `grad_stride` elements between token rows.
-zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* v, int64_t in_stride, const void* o,
-                   const float* lse, const void* d_o, float scale, void* dq, void* dk, void* dv, int64_t grad_stride,
-                   void* workspace, size_t workspace_bytes, void* stream) {
+// `phase` < 0: everything in one call.  Otherwise the first phase also clears the dQ accumulator and runs the
+// preprocess kernel, every phase runs the main kernel over its own kv groups, the last one also converts dQ.
+zl_status bwd_impl(const zl_tasks* t, int32_t phase, const void* q, const void* k, const void* v, int64_t in_stride,
+                   const void* o, const float* lse, const void* d_o, float scale, void* dq, void* dk, void* dv,
+                   int64_t grad_stride, void* workspace, size_t workspace_bytes, void* stream) {
     const Schedule& s = t->sched;
     if (s.tasks.empty()) return ZL_OK;
+    const int32_t n_phases = (int32_t)s.bwd_phase_begin.size() - 1;
+    if (phase >= n_phases) return ZL_ERR_INVALID_ARG;
+    const bool first = phase <= 0, last = phase < 0 || phase == n_phases - 1;
     if (t->device < 0) return ZL_ERR_CUDA;
     if (!on_handle_device(t)) return ZL_ERR_INVALID_ARG;
     if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !workspace) return ZL_ERR_INVALID_ARG;
@@ -474,11 +492,13 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
 
     BwdParams p{};
     p.tasks = t->d_tasks;
-    p.items = t->d_bwd_items;
+    const int32_t it0 = phase < 0 ? 0 : s.bwd_phase_begin[phase];
+    const int32_t it1 = phase < 0 ? (int32_t)s.bwd_items.size() : s.bwd_phase_begin[phase + 1];
+    p.items = t->d_bwd_items + it0;
     p.kv_groups = t->d_kv_groups;
     p.kv_group_tasks = t->d_kv_group_tasks;
     p.q_groups = t->d_q_groups;
-    p.n_items = (int32_t)s.bwd_items.size();
+    p.n_items = it1 - it0;
     p.n_q_groups = (int32_t)s.q_groups.size();
     p.n_heads = s.n_heads;
     p.total_q = s.total_q;
@@ -496,13 +516,13 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
     p.aug = ws + s.ws_aug_off;
     p.status = t->d_status;
 
-    if (cudaMemsetAsync(p.dq_acc, 0, (size_t)s.q_pad_total * s.n_heads * s.head_dim * sizeof(float), cs) != cudaSuccess)
-        return ZL_ERR_CUDA;
-    {
+    if (first) {
+        if (cudaMemsetAsync(p.dq_acc, 0, (size_t)s.q_pad_total * s.n_heads * s.head_dim * sizeof(float), cs) != cudaSuccess)
+            return ZL_ERR_CUDA;
         LaunchTimer lt(t, ZL_K_BWD_PRE, cs);
         if (launch_bwd_pre(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+        g_launches.fetch_add(1);
     }
-    g_launches.fetch_add(1);
     const bool pair = s.head_dim == 128 && (t->bwd_kernel == 2 || (t->bwd_kernel == 0 && kDefaultBwdPair));
     if (p.n_items > 0 && pair) {
         CUtensorMap tq64, tdo64, taug, tdq16;
@@ -512,8 +532,10 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
             !make_tmap_aug_rows(&taug, p.aug, (s.q_pad_total / kTileQ) * s.n_heads))
             return ZL_ERR_CUDA;
         BwdParams pp = p;
-        pp.items = t->d_bwd_pair_items;
-        pp.n_items = (int32_t)s.bwd_pair_items.size();
+        const int32_t pi0 = phase < 0 ? 0 : s.bwd_pair_phase_begin[phase];
+        const int32_t pi1 = phase < 0 ? (int32_t)s.bwd_pair_items.size() : s.bwd_pair_phase_begin[phase + 1];
+        pp.items = t->d_bwd_pair_items + pi0;
+        pp.n_items = pi1 - pi0;
         const int n_clusters = std::min<int>(t->n_sms / 2, pp.n_items);
         LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
         if (launch_bwd_pair(tq, tq64, tk, tv, tdo, tdo64, tdq16, taug, pp, n_clusters, cs) != cudaSuccess) return ZL_ERR_CUDA;
@@ -524,11 +546,11 @@ zl_status bwd_impl(const zl_tasks* t, const void* q, const void* k, const void* 
         if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, tdq, tdk, tdv, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
         g_launches.fetch_add(1);
     }
-    {
+    if (last) {
         LaunchTimer lt(t, ZL_K_BWD_POST, cs);
         if (launch_bwd_post(s.head_dim, p, t->n_sms, cs) != cudaSuccess) return ZL_ERR_CUDA;
+        g_launches.fetch_add(1);
     }
-    g_launches.fetch_add(1);
     return ZL_OK;
 }
 }  // namespace
@@ -540,7 +562,15 @@ zl_status zl_coalesced_attn_bwd(const zl_tasks* t, const void* q, const void* k,
                                 void* workspace, size_t workspace_bytes, void* stream) {
     if (!t) return ZL_ERR_INVALID_ARG;
     const int64_t hd = (int64_t)t->sched.n_heads * t->sched.head_dim;
-    return bwd_impl(t, q, k, v, hd, o, lse, d_o, scale, dq, dk, dv, hd, workspace, workspace_bytes, stream);
+    return bwd_impl(t, -1, q, k, v, hd, o, lse, d_o, scale, dq, dk, dv, hd, workspace, workspace_bytes, stream);
+}
+
+zl_status zl_coalesced_attn_bwd_phase(const zl_tasks* t, int32_t phase, const void* q, const void* k, const void* v,
+                                      const void* o, const float* lse, const void* d_o, float scale, void* dq, void* dk,
+                                      void* dv, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!t || phase < 0) return ZL_ERR_INVALID_ARG;
+    const int64_t hd = (int64_t)t->sched.n_heads * t->sched.head_dim;
+    return bwd_impl(t, phase, q, k, v, hd, o, lse, d_o, scale, dq, dk, dv, hd, workspace, workspace_bytes, stream);
 }
 
 zl_status zl_coalesced_attn_bwd_packed(const zl_tasks* t, const void* qkv, const void* o, const float* lse,
@@ -553,7 +583,7 @@ zl_status zl_coalesced_attn_bwd_packed(const zl_tasks* t, const void* qkv, const
     const int64_t hd = (int64_t)s.n_heads * s.head_dim;
     const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(qkv);
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(dqkv);
-    return bwd_impl(t, in, in + hd, in + 2 * hd, 3 * hd, o, lse, d_o, scale, out, out + hd, out + 2 * hd, 3 * hd,
+    return bwd_impl(t, -1, in, in + hd, in + 2 * hd, 3 * hd, o, lse, d_o, scale, out, out + hd, out + 2 * hd, 3 * hd,
                     workspace, workspace_bytes, stream);
 }
 
@@ -596,6 +626,94 @@ zl_status zl_coalesced_attn_bwd_noalloc(const zl_tasks* t, const void* q, const 
     return zl_coalesced_attn_bwd(t, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, ZL_NOALLOC_SCRATCH_BYTES, stream);
 }
 
+namespace {
+// Groups a work list by the phase of each item's unit (stable: the order inside a phase stays) and records
+// where each phase begins.
+void regroup_by_phase(std::vector<WorkItem>* items, const std::vector<int32_t>& unit_phase, int32_t n_phases,
+                      std::vector<int32_t>* begin) {
+    std::stable_sort(items->begin(), items->end(),
+                     [&](const WorkItem& a, const WorkItem& b) { return unit_phase[a.unit] < unit_phase[b.unit]; });
+    begin->assign((size_t)n_phases + 1, 0);
+    for (const WorkItem& w : *items) ++(*begin)[(size_t)unit_phase[w.unit] + 1];
+    for (int32_t i = 0; i < n_phases; ++i) (*begin)[(size_t)i + 1] += (*begin)[i];
+}
+
+// Per-task phases from the caller's per-sequence and per-shard arrays (NULL = phase 0); a task that stands for
+// several shards (fused chunks) takes the latest of their phases.
+zl_status task_phases(const Schedule& s, const int32_t* whole_phase, const int32_t* shard_phase, int32_t n_phases,
+                      std::vector<int32_t>* out) {
+    if (n_phases < 1 || n_phases > ZL_MAX_PHASES) return ZL_ERR_INVALID_ARG;
+    out->assign(s.tasks.size(), 0);
+    for (size_t i = 0; i < s.whole_to_task.size(); ++i) {
+        const int32_t ph = whole_phase ? whole_phase[i] : 0;
+        if (ph < 0 || ph >= n_phases) return ZL_ERR_INVALID_ARG;
+        if (s.whole_to_task[i] >= 0) (*out)[s.whole_to_task[i]] = std::max((*out)[s.whole_to_task[i]], ph);
+    }
+    for (size_t i = 0; i < s.shard_to_task.size(); ++i) {
+        const int32_t ph = shard_phase ? shard_phase[i] : 0;
+        if (ph < 0 || ph >= n_phases) return ZL_ERR_INVALID_ARG;
+        if (s.shard_to_task[i] >= 0) (*out)[s.shard_to_task[i]] = std::max((*out)[s.shard_to_task[i]], ph);
+    }
+    return ZL_OK;
+}
+
+zl_status upload_items(const zl_tasks* t, WorkItem* dst, const std::vector<WorkItem>& items, cudaStream_t cs) {
+    if (t->device < 0 || items.empty()) return ZL_OK;
+    if (cudaMemcpyAsync(dst, items.data(), items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaStreamSynchronize(cs) != cudaSuccess)
+        return ZL_ERR_CUDA;
+    return ZL_OK;
+}
+}  // namespace
+
+zl_status zl_set_fwd_phases(zl_tasks* t, const int32_t* whole_phase, const int32_t* shard_phase, int32_t n_phases,
+                            void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    if (t->device >= 0 && !on_handle_device(t)) return ZL_ERR_INVALID_ARG;
+    Schedule& s = t->sched;
+    std::vector<int32_t> ph;
+    const zl_status st = task_phases(s, whole_phase, shard_phase, n_phases, &ph);
+    if (st != ZL_OK) return st;
+    s.fwd_task_phase = ph;
+    regroup_by_phase(&s.fwd_items, s.fwd_task_phase, n_phases, &s.fwd_phase_begin);
+    return upload_items(t, t->d_fwd_items, s.fwd_items, static_cast<cudaStream_t>(stream));
+}
+
+zl_status zl_set_bwd_phases(zl_tasks* t, const int32_t* whole_phase, const int32_t* shard_phase, int32_t n_phases,
+                            void* stream) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    if (t->device >= 0 && !on_handle_device(t)) return ZL_ERR_INVALID_ARG;
+    Schedule& s = t->sched;
+    std::vector<int32_t> ph;
+    const zl_status st = task_phases(s, whole_phase, shard_phase, n_phases, &ph);
+    if (st != ZL_OK) return st;
+    // a kv group is finished by one work item, so it runs in the latest phase any of its tasks asks for
+    s.bwd_group_phase.assign(s.kv_groups.size(), 0);
+    for (size_t g = 0; g < s.kv_groups.size(); ++g)
+        for (int32_t j = 0; j < s.kv_groups[g].n_tasks; ++j)
+            s.bwd_group_phase[g] = std::max(s.bwd_group_phase[g], ph[s.kv_group_tasks[s.kv_groups[g].task_begin + j]]);
+    regroup_by_phase(&s.bwd_items, s.bwd_group_phase, n_phases, &s.bwd_phase_begin);
+    regroup_by_phase(&s.bwd_pair_items, s.bwd_group_phase, n_phases, &s.bwd_pair_phase_begin);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const zl_status st1 = upload_items(t, t->d_bwd_items, s.bwd_items, cs);
+    if (st1 != ZL_OK) return st1;
+    return upload_items(t, t->d_bwd_pair_items, s.bwd_pair_items, cs);
+}
+
+zl_status zl_phase_info(const zl_tasks* t, int32_t* n_fwd_phases, int32_t* n_bwd_phases, int32_t* fwd_items_per_phase,
+                        int32_t* bwd_items_per_phase) {
+    if (!t) return ZL_ERR_INVALID_ARG;
+    const Schedule& s = t->sched;
+    const int32_t nf = (int32_t)s.fwd_phase_begin.size() - 1, nb = (int32_t)s.bwd_phase_begin.size() - 1;
+    if (n_fwd_phases) *n_fwd_phases = nf;
+    if (n_bwd_phases) *n_bwd_phases = nb;
+    if (fwd_items_per_phase)
+        for (int32_t i = 0; i < nf; ++i) fwd_items_per_phase[i] = s.fwd_phase_begin[i + 1] - s.fwd_phase_begin[i];
+    if (bwd_items_per_phase)
+        for (int32_t i = 0; i < nb; ++i) bwd_items_per_phase[i] = s.bwd_phase_begin[i + 1] - s.bwd_phase_begin[i];
+    return ZL_OK;
+}
+
 zl_status zl_debug_set_fwd_order(zl_tasks* t, int32_t mode, void* stream) {
     if (!t || mode < 0 || mode > 2) return ZL_ERR_INVALID_ARG;
     Schedule& s = t->sched;
@@ -611,13 +729,9 @@ zl_status zl_debug_set_fwd_order(zl_tasks* t, int32_t mode, void* stream) {
             return false;
         });
     }
-    if (t->device < 0 || s.fwd_items.empty()) return ZL_OK;
-    cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(t->d_fwd_items, s.fwd_items.data(), s.fwd_items.size() * sizeof(WorkItem),
-                        cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-        cudaStreamSynchronize(cs) != cudaSuccess)
-        return ZL_ERR_CUDA;
-    return ZL_OK;
+    // the list stays grouped by launch phase
+    regroup_by_phase(&s.fwd_items, s.fwd_task_phase, (int32_t)s.fwd_phase_begin.size() - 1, &s.fwd_phase_begin);
+    return upload_items(t, t->d_fwd_items, s.fwd_items, static_cast<cudaStream_t>(stream));
 }
 
 zl_status zl_set_bwd_kernel(zl_tasks* t, int32_t kernel) {

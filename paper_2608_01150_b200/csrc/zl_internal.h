@@ -62,6 +62,7 @@ struct Schedule {
     int32_t n_heads = 0, head_dim = 0, total_q = 0, total_kv = 0;
     std::vector<Task> tasks;
     std::vector<int32_t> task_head_begin, task_head_count;  // per task (host only: items carry their head)
+    std::vector<int32_t> whole_to_task;     // per input whole sequence: task index or -1 (empty sequence)
     std::vector<int32_t> shard_to_task;     // per input shard: task index or -1 (q_len == 0)
     std::vector<int32_t> shard_slot_off;    // per input shard: slot row offset (or 0)
     std::vector<int32_t> shard_slot_rows;   // per input shard: padded slot rows (0 if skipped)
@@ -75,6 +76,10 @@ struct Schedule {
     std::vector<WorkItem> fwd_items;
     std::vector<WorkItem> bwd_items;
     std::vector<WorkItem> bwd_pair_items;   // (kv group, head, first key row, rows <= 256): two key tiles per CTA pair
+    // Launch phases: the work lists are grouped by phase and a phased launch walks one group.  Forward phases are
+    // per task, backward phases per kv group; one phase (the whole list) until zl_set_fwd_phases / zl_set_bwd_phases.
+    std::vector<int32_t> fwd_task_phase, bwd_group_phase;
+    std::vector<int32_t> fwd_phase_begin, bwd_phase_begin, bwd_pair_phase_begin;  // n_phases + 1 offsets into the lists
     int64_t partial_rows = 0;
     int32_t n_fused_ranges = 0;             // shard query ranges lowered to one final task (chunk fusion)
     size_t bwd_workspace_bytes = 0;

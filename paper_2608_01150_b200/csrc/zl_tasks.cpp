@@ -144,6 +144,7 @@ zl_status build_schedule(const std::vector<InputTask>& in, int32_t n_shards, int
     }
 
     // ---- tasks: whole sequences in placement order, then shards in the caller's order
+    s->whole_to_task.clear();
     s->shard_to_task.assign(n_shards, -1);
     s->shard_slot_off.assign(n_shards, 0);
     s->shard_slot_rows.assign(n_shards, 0);
@@ -156,6 +157,7 @@ zl_status build_schedule(const std::vector<InputTask>& in, int32_t n_shards, int
         s->task_head_count.push_back(src.head_count);
     };
     for (size_t i = 0; i < n_in; ++i) {
+        if (in[i].shard_idx < 0) s->whole_to_task.push_back(live[i] ? (int32_t)s->tasks.size() : -1);
         if (!live[i]) continue;
         const InputTask& d = in[i];
         Task t{};
@@ -293,6 +295,13 @@ zl_status build_schedule(const std::vector<InputTask>& in, int32_t n_shards, int
                 s->bwd_pair_items.push_back({(int32_t)g, h, r, std::min(2 * kTileKV, s->kv_groups[g].kv_len - r)});
     }
     std::stable_sort(s->bwd_pair_items.begin(), s->bwd_pair_items.end(), bwd_order);
+
+    // one launch phase until the caller says otherwise
+    s->fwd_task_phase.assign(s->tasks.size(), 0);
+    s->bwd_group_phase.assign(s->kv_groups.size(), 0);
+    s->fwd_phase_begin = {0, (int32_t)s->fwd_items.size()};
+    s->bwd_phase_begin = {0, (int32_t)s->bwd_items.size()};
+    s->bwd_pair_phase_begin = {0, (int32_t)s->bwd_pair_items.size()};
 
     // backward workspace over the padded query slots: fp32 dQ accumulator [q_pad, H, d], then one
     // 4 KB "augmentation" tile per (head, 128-row query tile) holding -LSE/scale and -D split

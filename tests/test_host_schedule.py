@@ -282,3 +282,83 @@ def test_head_range_validation(Z):
     # the same token ranges on disjoint head ranges are independent tasks
     h = build([(0, 100, 0, 4)], [(100, 50, 100, 50, 0, 0, 2), (100, 50, 100, 50, 0, 2, 2)])
     assert h.info.n_tasks == 3 and h.info.n_merge_groups == 2
+
+
+# ------------------------------------------------------------------------------------------------ launch phases
+def _phase_placement():
+    # two whole sequences + one query chunk against four K/V chunks, 2 heads
+    return W.make_placement("ph", 2, 64, 0, [300, 700], [(1, 4, 500)])
+
+
+def test_a_handle_starts_with_one_phase_per_direction(Z):
+    h = _build(Z, _phase_placement())
+    fi, bi = h.phase_info()
+    assert fi == [h.info.n_fwd_items] and bi == [h.info.n_bwd_items]
+
+
+def test_forward_phases_regroup_the_list_and_keep_longest_first_inside_a_phase(Z):
+    p = _phase_placement()
+    h = _build(Z, p)
+    tasks = _tasks_of(p)
+    before = sorted(h.fwd_items())
+    h.set_fwd_phases([0, 0], [0, 1, 2, 3], 4)
+    fi, _ = h.phase_info()
+    items = h.fwd_items()
+    assert sorted(items) == before and sum(fi) == len(items)
+    # tasks 0,1 are the whole sequences, 2..5 the shards in the caller's order
+    phase_of_task = {0: 0, 1: 0, 2: 0, 3: 1, 4: 2, 5: 3}
+    pos = 0
+    for ph, n in enumerate(fi):
+        chunk = items[pos:pos + n]
+        assert n > 0 and all(phase_of_task[t] == ph for (t, _, _, _) in chunk)
+        keys = [(tasks[t][3], rows) for (t, _, _, rows) in chunk]
+        assert all(keys[i] >= keys[i + 1] for i in range(len(keys) - 1))
+        pos += n
+    # changing the order inside the list keeps the grouping
+    h.set_fwd_order(2)
+    assert h.phase_info()[0] == fi
+    items2 = h.fwd_items()
+    assert all(phase_of_task[t] == 0 for (t, _, _, _) in items2[:fi[0]])
+    # one phase again
+    h.set_fwd_phases(None, None, 1)
+    assert h.phase_info()[0] == [len(items)]
+
+
+def test_backward_phases_follow_the_kv_group_with_the_latest_phase(Z):
+    # kv range A serves two query chunks, kv range B one; an image of 200
+    p = W.custom_placement("c", 1, 64, 0, [0, 200],
+                           [(200, 300, 200, 256, 0), (500, 300, 200, 256, 1), (200, 300, 456, 256, 0)], 800, 712)
+    h = _build(Z, p)
+    n = h.info.n_bwd_items
+    # the two tasks on kv range A ask for phases 0 and 1: the group runs in phase 1
+    h.set_bwd_phases([1], [0, 1, 0], 2)
+    _, bi = h.phase_info()
+    assert sum(bi) == n
+    items = h.bwd_items()
+    groups_phase0 = {g for (g, _, _, _) in items[:bi[0]]}
+    groups_phase1 = {g for (g, _, _, _) in items[bi[0]:]}
+    assert len(groups_phase0) == 1 and len(groups_phase1) == 2 and not (groups_phase0 & groups_phase1)
+    assert bi[0] == 2      # kv range B: 256 rows = two key tiles, one head
+
+
+def test_phase_arguments_are_validated(Z):
+    h = _build(Z, _phase_placement())
+    for bad in ([0, 0], [0, 0, 0, 4]), ([0, -1], [0, 0, 0, 0]):
+        with pytest.raises(Z.ZlError, match="ZL_ERR_INVALID_ARG"):
+            h.set_fwd_phases(bad[0], bad[1], 4)
+    for n_phases in (0, Z.MAX_PHASES + 1):
+        with pytest.raises(Z.ZlError, match="ZL_ERR_INVALID_ARG"):
+            h.set_bwd_phases(None, None, n_phases)
+    # a failed call leaves the handle as it was
+    assert h.phase_info()[0] == [h.info.n_fwd_items]
+
+
+def test_a_fused_range_runs_in_the_latest_phase_of_its_chunks(Z):
+    p = _phase_placement()
+    h = Z.build_tasks(p.cu_seqlens, p.shards, p.total_q, p.total_kv, p.n_heads, p.head_dim,
+                      flags=Z.BUILD_FUSE_LOCAL_CHUNKS)
+    assert h.info.n_fused_ranges == 1 and h.info.n_tasks == 3
+    h.set_fwd_phases(None, [0, 1, 2, 1], 3)
+    fi, _ = h.phase_info()
+    assert fi[1] == 0 and fi[2] > 0 and fi[0] > 0
+    assert all(t == 2 for (t, _, _, _) in h.fwd_items()[fi[0]:])
