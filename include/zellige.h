@@ -355,6 +355,11 @@ zl_status zl_debug_set_fwd_order(zl_tasks* tasks, int32_t mode, void* stream);
  * (head_dim 128 only: ZL_ERR_UNSUPPORTED otherwise).  Results agree within the gradient tolerance; dK
  * and dV of the two kernels may differ in the last bit (different accumulation order). */
 zl_status zl_set_bwd_kernel(zl_tasks* tasks, int32_t kernel);
+/* zl_set_sm_margin: the persistent kernels (forward, backward main) of this handle leave `n_sms` of the GPU's SMs
+ * without a CTA (at least two SMs are always used), so that kernels of another stream -- the collectives that
+ * run beside a launch phase -- find a free SM instead of waiting for the launch to end.  0 (the default) uses
+ * every SM.  Results do not depend on it.  (No paper counterpart.) */
+zl_status zl_set_sm_margin(zl_tasks* tasks, int32_t n_sms);
 zl_status zl_selftest_bounded_wait(const zl_tasks* tasks, int32_t limit_us, void* stream);
 
 const char* zl_status_str(zl_status s);

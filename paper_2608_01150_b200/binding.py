@@ -96,6 +96,8 @@ def _load():
                                                 ctypes.c_size_t, vp]
     lib.zl_phase_info.restype = ctypes.c_int
     lib.zl_phase_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.zl_set_sm_margin.restype = ctypes.c_int
+    lib.zl_set_sm_margin.argtypes = [vp, i32]
     lib.zl_coalesced_attn_bwd_noalloc.restype = ctypes.c_int
     lib.zl_coalesced_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.zl_last_device_status.restype = ctypes.c_int
@@ -224,6 +226,10 @@ class TaskHandle:
         fi, bi = (ctypes.c_int32 * MAX_PHASES)(), (ctypes.c_int32 * MAX_PHASES)()
         _check(_lib.zl_phase_info(self._ptr, ctypes.byref(nf), ctypes.byref(nb), fi, bi), "zl_phase_info")
         return list(fi[:nf.value]), list(bi[:nb.value])
+
+    def set_sm_margin(self, n_sms: int):
+        """zl_set_sm_margin: SMs the persistent kernels leave free for kernels of other streams."""
+        _check(_lib.zl_set_sm_margin(self._ptr, n_sms), "zl_set_sm_margin")
 
     def set_bwd_kernel(self, kernel: int):
         """0 library default, 1 one CTA per key tile, 2 CTA pairs (head_dim 128)."""

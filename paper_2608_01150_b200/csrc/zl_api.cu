@@ -25,6 +25,7 @@ struct zl_tasks {
     WorkItem* d_bwd_items = nullptr;
     WorkItem* d_bwd_pair_items = nullptr;
     int bwd_kernel = 0;           // 0: library default, 1: one CTA per key tile, 2: CTA pairs (head_dim 128)
+    int sm_margin = 0;            // SMs the persistent kernels leave free (for communication kernels running beside them)
     MergeGroup* d_merge_groups = nullptr;
     int32_t* d_merge_parts = nullptr;
     int32_t* d_merge_prefix = nullptr;
@@ -382,7 +383,7 @@ zl_status fwd_impl(const zl_tasks* t, int32_t phase, const void* q, const void* 
     p.o_partial = o_partial;
     p.lse_partial = lse_partial;
     p.status = t->d_status;
-    const int grid = std::min<int>(t->n_sms, p.n_items);
+    const int grid = std::min<int>(std::max(2, t->n_sms - t->sm_margin), p.n_items);
     {
         LaunchTimer lt(t, ZL_K_FWD, static_cast<cudaStream_t>(stream));
         if (launch_fwd(s.head_dim, tq, tk, tv, to, top, p, grid, static_cast<cudaStream_t>(stream)) != cudaSuccess)
@@ -536,12 +537,12 @@ zl_status bwd_impl(const zl_tasks* t, int32_t phase, const void* q, const void* 
         const int32_t pi1 = phase < 0 ? (int32_t)s.bwd_pair_items.size() : s.bwd_pair_phase_begin[phase + 1];
         pp.items = t->d_bwd_pair_items + pi0;
         pp.n_items = pi1 - pi0;
-        const int n_clusters = std::min<int>(t->n_sms / 2, pp.n_items);
+        const int n_clusters = std::min<int>(std::max(2, t->n_sms - t->sm_margin) / 2, pp.n_items);
         LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
         if (launch_bwd_pair(tq, tq64, tk, tv, tdo, tdo64, tdq16, taug, pp, n_clusters, cs) != cudaSuccess) return ZL_ERR_CUDA;
         g_launches.fetch_add(1);
     } else if (p.n_items > 0) {
-        const int grid = std::min<int>(t->n_sms, p.n_items);
+        const int grid = std::min<int>(std::max(2, t->n_sms - t->sm_margin), p.n_items);
         LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
         if (launch_bwd_main(s.head_dim, tq, tk, tv, tdo, tdq, tdk, tdv, p, grid, cs) != cudaSuccess) return ZL_ERR_CUDA;
         g_launches.fetch_add(1);
@@ -732,6 +733,12 @@ zl_status zl_debug_set_fwd_order(zl_tasks* t, int32_t mode, void* stream) {
     // the list stays grouped by launch phase
     regroup_by_phase(&s.fwd_items, s.fwd_task_phase, (int32_t)s.fwd_phase_begin.size() - 1, &s.fwd_phase_begin);
     return upload_items(t, t->d_fwd_items, s.fwd_items, static_cast<cudaStream_t>(stream));
+}
+
+zl_status zl_set_sm_margin(zl_tasks* t, int32_t n_sms) {
+    if (!t || n_sms < 0) return ZL_ERR_INVALID_ARG;
+    t->sm_margin = n_sms;
+    return ZL_OK;
 }
 
 zl_status zl_set_bwd_kernel(zl_tasks* t, int32_t kernel) {

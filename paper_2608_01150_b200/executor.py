@@ -21,6 +21,14 @@ configuration):
            n_heads/h heads, one inverse all-to-all returns the outputs.  Ulysses sequences that
            share configuration and rank set are batched into one all-to-all each way.
 
+Overlap (Section IV-D): with a phased attention step (an object with fwd_begin / fwd_phase / fwd_end
+and bwd_begin / bwd_phase / bwd_end, see :class:`EngineAttention`) the tasks whose K/V are already local
+are launched first and the collectives run beside them on a second stream; every arrival -- the
+gathered chunks of an all-gather segment, the chunk of each ring step, the sequences of a Ulysses
+batch -- releases the launch phase of the tasks that were waiting for it.  In the backward the
+gradients of remote K/V chunks are computed first and travel to their owners (reduce-scatter) while
+the rest of the backward runs.
+
 The attention step itself is a pair of callables, so that the executor is plumbing only:
 :class:`EngineAttention` (below) binds it to the CUDA library; tests bind it to a checker.  The
 kernels only ever see this GPU's memory: K/V chunks of other ranks are first moved into local
@@ -34,6 +42,7 @@ from typing import Callable, Dict, List, Optional, Sequence, Tuple
 import torch
 
 ALL_GATHER, RING, ULYSSES, WHOLE = "all_gather", "ring", "ulysses", "whole"
+MAX_PHASES = 64  # launch phases of one handle (ZL_MAX_PHASES of the C ABI)
 
 
 @dataclass(frozen=True)
@@ -155,6 +164,16 @@ class RankSchedule:
     heads: Dict[int, Tuple[int, int]] = field(default_factory=dict)           # seg -> (head_begin, head_count)
     order: List[int] = field(default_factory=list)                            # this rank's segments in collective order
     ulysses_batches: List[List[int]] = field(default_factory=list)            # segment indices batched per all-to-all
+    # launch phases (phase 0 = runnable before any collective); indices follow `whole` and `shards`
+    fwd_whole_phase: List[int] = field(default_factory=list)
+    fwd_shard_phase: List[int] = field(default_factory=list)
+    n_fwd_phases: int = 1
+    bwd_whole_phase: List[int] = field(default_factory=list)
+    bwd_shard_phase: List[int] = field(default_factory=list)
+    n_bwd_phases: int = 1
+    whole_index: Dict[int, int] = field(default_factory=dict)                 # seg -> index into `whole`
+    shard_index: Dict[int, List[int]] = field(default_factory=dict)           # seg -> index into `shards` per chunk
+    arrival_phase: Dict[int, List[int]] = field(default_factory=dict)         # seg -> forward phase per chunk (CP) / [phase] (Ulysses)
 
 
 def lower(segments: Sequence[Segment], rank: int, world_size: int, n_heads: int) -> RankSchedule:
@@ -183,6 +202,7 @@ def lower(segments: Sequence[Segment], rank: int, world_size: int, n_heads: int)
             hb = s.ranks.index(rank) * hc
         else:
             continue
+        sch.whole_index[i] = len(sch.whole)
         sch.whole.append((row, s.length, hb, hc))
         sch.q_rows[i] = (row, s.length)
         sch.kv_rows[i] = (row, s.length)
@@ -200,9 +220,11 @@ def lower(segments: Sequence[Segment], rank: int, world_size: int, n_heads: int)
         sch.kv_rows[i] = (kv_row, s.length)
         sch.heads[i] = (0, n_heads)
         chunks = []
+        sch.shard_index[i] = []
         for j in range(s.degree):
             ca, cb = chunk_bounds(s.length, s.degree, j)
             chunks.append((kv_row + ca, cb - ca))
+            sch.shard_index[i].append(len(sch.shards))
             sch.shards.append((q_row, b - a, kv_row + ca, cb - ca, s.seq_id))
         sch.chunk_rows[i] = chunks
         q_row += b - a
@@ -215,6 +237,51 @@ def lower(segments: Sequence[Segment], rank: int, world_size: int, n_heads: int)
         if s.kind == ULYSSES:
             batches.setdefault((s.config, s.ranks), []).append(i)
     sch.ulysses_batches = list(batches.values())
+    # ---- launch phases, numbered in the order the collectives deliver: forward phase 0 holds the whole sequences
+    # and every context-parallel query chunk against its own K/V chunk
+    sch.fwd_whole_phase, sch.fwd_shard_phase = [0] * len(sch.whole), [0] * len(sch.shards)
+    sch.bwd_whole_phase, sch.bwd_shard_phase = [0] * len(sch.whole), [0] * len(sch.shards)
+    phase, seen_batches = 0, set()
+
+    def next_phase():
+        nonlocal phase
+        phase = min(phase + 1, MAX_PHASES - 1)
+        return phase
+
+    for i in mine:
+        s = segments[i]
+        if s.kind == WHOLE:
+            continue
+        if s.kind == ULYSSES:
+            bi = next(n for n, b in enumerate(sch.ulysses_batches) if i in b)
+            if bi in seen_batches:
+                continue
+            seen_batches.add(bi)
+            ph = next_phase()
+            for j in sch.ulysses_batches[bi]:
+                sch.fwd_whole_phase[sch.whole_index[j]] = ph
+                sch.arrival_phase[j] = [ph]
+            continue
+        k, pos = s.degree, s.ranks.index(rank)
+        per_chunk = [0] * k
+        if s.kind == ALL_GATHER:
+            ph = next_phase()
+            per_chunk = [0 if j == pos else ph for j in range(k)]
+        else:
+            for t in range(1, k):                      # ring step t delivers the chunk of the rank t places back
+                per_chunk[(pos - t) % k] = next_phase()
+        sch.arrival_phase[i] = per_chunk
+        for j in range(k):
+            sch.fwd_shard_phase[sch.shard_index[i][j]] = per_chunk[j]
+    sch.n_fwd_phases = phase + 1
+    # backward: gradients of remote K/V chunks first (phase 0), everything else after (phase 1)
+    if sch.shards:
+        sch.n_bwd_phases = 2
+        sch.bwd_whole_phase = [1] * len(sch.whole)
+        for i, idx in sch.shard_index.items():
+            pos = segments[i].ranks.index(rank)
+            for j, si in enumerate(idx):
+                sch.bwd_shard_phase[si] = 1 if j == pos else 0
     return sch
 
 
@@ -248,7 +315,9 @@ class CPExecutor:
         self.cache.ensure(self.segments)
         self.schedule = lower(self.segments, self.rank, self.world_size, n_heads)
         self.log: List[Tuple] = []
+        self.phase_log: List[int] = []
         self._saved = None
+        self._comm_stream = None
 
     # ---- helpers
     def _piece(self, seg_index: int) -> LocalPiece:
@@ -357,9 +426,12 @@ class CPExecutor:
         return parts.permute(1, 2, 0, 3, 4).reshape(rows_of_rank[pos], C, self.n_heads, self.head_dim)
 
     # ---- forward
-    def forward(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, attn_fwd: AttnFwd) -> torch.Tensor:
+    def forward(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, attn_fwd) -> torch.Tensor:
+        """`attn_fwd`: a callable (one launch after all collectives) or a phased attention step (overlap)."""
         sch, H, d = self.schedule, self.n_heads, self.head_dim
         assert q.shape == (sch.own_tokens, H, d) and k.shape == q.shape and v.shape == q.shape
+        if hasattr(attn_fwd, "fwd_phase"):
+            return self._forward_phased(q, k, v, attn_fwd)
         Q = torch.zeros((sch.total_q, H, d), dtype=q.dtype, device=q.device)
         K = torch.zeros((sch.total_kv, H, d), dtype=q.dtype, device=q.device)
         V = torch.zeros_like(K)
@@ -427,10 +499,174 @@ class CPExecutor:
                 pos += n
         return out
 
+    # ---- overlap: launch phases under the collectives
+    def _streams(self, ref: torch.Tensor):
+        """(compute stream, communication stream) on CUDA, (None, None) on CPU."""
+        if not ref.is_cuda:
+            return None, None
+        if self._comm_stream is None:
+            self._comm_stream = torch.cuda.Stream(device=ref.device)
+        return torch.cuda.current_stream(ref.device), self._comm_stream
+
+    class _On:
+        """`with _On(stream):` -- torch.cuda.stream(stream), or nothing on CPU."""
+        def __init__(self, stream):
+            self.ctx = torch.cuda.stream(stream) if stream is not None else None
+
+        def __enter__(self):
+            if self.ctx is not None:
+                self.ctx.__enter__()
+
+        def __exit__(self, *a):
+            if self.ctx is not None:
+                self.ctx.__exit__(*a)
+
+    def _release(self, main, comm, fn):
+        """Runs `fn` (a launch on the compute stream) after everything issued so far on the communication stream."""
+        if comm is not None:
+            ev = torch.cuda.Event()
+            ev.record(comm)
+            main.wait_event(ev)
+        fn()
+
+    def _forward_phased(self, q, k, v, attn) -> torch.Tensor:
+        sch, H, d = self.schedule, self.n_heads, self.head_dim
+        Q = torch.zeros((sch.total_q, H, d), dtype=q.dtype, device=q.device)
+        K = torch.zeros((sch.total_kv, H, d), dtype=q.dtype, device=q.device)   # zero-filled: rows in flight stay finite
+        V = torch.zeros_like(K)
+        main, comm = self._streams(q)
+        self.log = []
+        # 1. everything that needs no communication
+        for i in sch.order:
+            s, pc = self.segments[i], self._piece(i)
+            own = slice(pc.own_off, pc.own_off + pc.g1 - pc.g0)
+            if s.kind == WHOLE:
+                qo, ql = sch.q_rows[i]
+                Q[qo:qo + ql], K[qo:qo + ql], V[qo:qo + ql] = q[own], k[own], v[own]
+            elif s.kind in (ALL_GATHER, RING):
+                qo, ql = sch.q_rows[i]
+                Q[qo:qo + ql] = q[own]
+                co, cl = sch.chunk_rows[i][s.ranks.index(self.rank)]
+                K[co:co + cl], V[co:co + cl] = k[own], v[own]
+        if comm is not None:
+            comm.wait_stream(main)
+            for t in (Q, K, V, q, k, v):
+                t.record_stream(comm)
+        st = attn.fwd_begin(sch, Q, K, V)
+        attn.fwd_phase(sch, st, 0)
+        self.phase_log = [0]
+
+        def launch(ph):
+            if ph not in self.phase_log:          # phases are capped at MAX_PHASES: the last one may be shared
+                self.phase_log.append(ph)
+                self._release(main, comm, lambda: attn.fwd_phase(sch, st, ph))
+
+        # 2. the collectives, in the common order, on the communication stream; each arrival releases its phase
+        done_batches = set()
+        for i in sch.order:
+            s, pc = self.segments[i], self._piece(i)
+            own = slice(pc.own_off, pc.own_off + pc.g1 - pc.g0)
+            if s.kind == WHOLE:
+                continue
+            if s.kind == ALL_GATHER:
+                self.log.append((s.kind, s.seq_id, tuple(s.ranks)))
+                with self._On(comm):
+                    self._all_gather_chunks(K, sch.chunk_rows[i], k[own], s)
+                    self._all_gather_chunks(V, sch.chunk_rows[i], v[own], s)
+                launch(max(sch.arrival_phase[i]))
+            elif s.kind == RING:
+                self.log.append((s.kind, s.seq_id, tuple(s.ranks)))
+                self._ring_gather_kv(K, V, sch.chunk_rows[i], s, comm,
+                                     lambda j, i=i: launch(sch.arrival_phase[i][j]))
+            else:
+                bi = next(n for n, b in enumerate(sch.ulysses_batches) if i in b)
+                if bi in done_batches:
+                    continue
+                done_batches.add(bi)
+                batch = sch.ulysses_batches[bi]
+                self.log.append(("ulysses_all_to_all", tuple(self.segments[j].seq_id for j in batch), tuple(s.ranks)))
+                with self._On(comm):
+                    rows = torch.cat([torch.arange(self._piece(j).own_off, self._piece(j).own_off + self._piece(j).g1 - self._piece(j).g0)
+                                      for j in batch]).to(q.device)
+                    packed = torch.stack([q[rows], k[rows], v[rows]], dim=1)
+                    full = self._ulysses_exchange(batch, packed, inverse=False)
+                    for j, f in zip(batch, full):
+                        (ro, rl), (hb, hc) = sch.q_rows[j], sch.heads[j]
+                        Q[ro:ro + rl, hb:hb + hc], K[ro:ro + rl, hb:hb + hc], V[ro:ro + rl, hb:hb + hc] = f[:, 0], f[:, 1], f[:, 2]
+                launch(sch.arrival_phase[i][0])
+        assert sorted(self.phase_log) == list(range(sch.n_fwd_phases)), (self.phase_log, sch.n_fwd_phases)
+        O, saved = attn.fwd_end(sch, st)
+        self._saved = (saved, Q.shape, K.shape)
+        return self._scatter_q_space(O, q.dtype, q.device, tag="ulysses_inverse_all_to_all")
+
+    def _ring_gather_kv(self, K, V, chunks, seg: Segment, comm, arrived):
+        """The ring of _ring_gather for K and V together; `arrived(j)` is called when chunk j is in place."""
+        group = self.cache.get(seg.ranks)
+        k, pos = seg.degree, seg.ranks.index(self.rank)
+        nxt, prv = seg.ranks[(pos + 1) % k], seg.ranks[(pos - 1) % k]
+        for t in range(1, k):
+            send_j, recv_j = (pos - t + 1) % k, (pos - t) % k
+            (so, sl), (ro, rl) = chunks[send_j], chunks[recv_j]
+            with self._On(comm):
+                recv_k, recv_v = torch.empty_like(K[ro:ro + rl]), torch.empty_like(V[ro:ro + rl])
+                ops = [self.dist.P2POp(self.dist.isend, K[so:so + sl].contiguous(), nxt, group=group),
+                       self.dist.P2POp(self.dist.isend, V[so:so + sl].contiguous(), nxt, group=group),
+                       self.dist.P2POp(self.dist.irecv, recv_k, prv, group=group),
+                       self.dist.P2POp(self.dist.irecv, recv_v, prv, group=group)]
+                for w in self.dist.batch_isend_irecv(ops):
+                    w.wait()
+                K[ro:ro + rl].copy_(recv_k)
+                V[ro:ro + rl].copy_(recv_v)
+            arrived(recv_j)
+
+    def _backward_phased(self, attn, saved, dO, early):
+        """Phase 0 computes dK/dV of the remote chunks; their reduce-scatter runs on the communication stream
+        while phase 1 computes the rest.  `early[seg]` receives what the other ranks contributed to this rank's
+        own chunk (the rank's own contribution is a result of phase 1 and is added by the caller)."""
+        sch = self.schedule
+        main, comm = self._streams(dO)
+        st = attn.bwd_begin(sch, saved, dO)
+        attn.bwd_phase(sch, st, 0)
+        dK, dV = attn.bwd_grads(st)
+        # snapshot of the remote chunks' gradients with zeros in the own chunk: phase 1 writes the own chunk while
+        # the collective reads
+        staged = {}
+        for i in sch.order:
+            s = self.segments[i]
+            if s.kind not in (ALL_GATHER, RING):
+                continue
+            a, b = sch.kv_rows[i][0], sch.kv_rows[i][0] + sch.kv_rows[i][1]
+            co, cl = sch.chunk_rows[i][s.ranks.index(self.rank)]
+            sk, sv = dK[a:b].clone(), dV[a:b].clone()
+            sk[co - a:co - a + cl] = 0
+            sv[co - a:co - a + cl] = 0
+            staged[i] = (sk, sv, a)
+        if comm is not None:
+            comm.wait_stream(main)
+            for sk, sv, _ in staged.values():
+                sk.record_stream(comm)
+                sv.record_stream(comm)
+        attn.bwd_phase(sch, st, 1)
+        for i in sch.order:
+            if i not in staged:
+                continue
+            s = self.segments[i]
+            sk, sv, a = staged[i]
+            rel = [(off - a, ln) for off, ln in sch.chunk_rows[i]]
+            self.log.append(("reduce_scatter", s.seq_id, tuple(s.ranks)))
+            with self._On(comm):
+                early[i] = (self._reduce_scatter_chunks(sk, rel, s), self._reduce_scatter_chunks(sv, rel, s))
+        out = attn.bwd_end(sch, st)
+        if comm is not None:
+            main.wait_stream(comm)
+        return out
+
     # ---- backward
-    def backward(self, d_o: torch.Tensor, attn_bwd: AttnBwd) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    def backward(self, d_o: torch.Tensor, attn_bwd) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+        """`attn_bwd`: a callable, or a phased attention step (gradients of remote chunks leave early)."""
         sch, H, d = self.schedule, self.n_heads, self.head_dim
         saved, q_shape, k_shape = self._saved
+        phased = hasattr(attn_bwd, "bwd_phase") and sch.n_bwd_phases == 2
         dO = torch.zeros(q_shape, dtype=d_o.dtype, device=d_o.device)
         self.log = []
         done_batches = set()
@@ -453,9 +689,17 @@ class CPExecutor:
             for j, f in zip(batch, full):
                 (ro, rl), (hb, hc) = sch.q_rows[j], sch.heads[j]
                 dO[ro:ro + rl, hb:hb + hc] = f[:, 0]
-        dQ, dK, dV = attn_bwd(sch, saved, dO)
         dq = torch.zeros((sch.own_tokens, H, d), dtype=d_o.dtype, device=d_o.device)
         dk, dv = torch.zeros_like(dq), torch.zeros_like(dq)
+        early: Dict[int, Tuple[torch.Tensor, torch.Tensor]] = {}
+        if phased:
+            dQ, dK, dV = self._backward_phased(attn_bwd, saved, dO, early)
+        elif hasattr(attn_bwd, "bwd_phase"):      # a phased step on a rank without remote chunks: one phase
+            st = attn_bwd.bwd_begin(sch, saved, dO)
+            attn_bwd.bwd_phase(sch, st, 0)
+            dQ, dK, dV = attn_bwd.bwd_end(sch, st)
+        else:
+            dQ, dK, dV = attn_bwd(sch, saved, dO)
         done_batches = set()
         for i in sch.order:
             s, pc = self.segments[i], self._piece(i)
@@ -465,6 +709,11 @@ class CPExecutor:
                 dq[own], dk[own], dv[own] = dQ[qo:qo + ql], dK[qo:qo + ql], dV[qo:qo + ql]
             elif s.kind in (ALL_GATHER, RING):
                 dq[own] = dQ[qo:qo + ql]
+                if i in early:
+                    # the other ranks' contributions arrived under the second phase; add this rank's own
+                    co, cl = sch.chunk_rows[i][s.ranks.index(self.rank)]
+                    dk[own], dv[own] = early[i][0] + dK[co:co + cl], early[i][1] + dV[co:co + cl]
+                    continue
                 # every rank holds the gradient of ALL chunks with respect to its own queries: sum them at the owners
                 self.log.append(("reduce_scatter", s.seq_id, tuple(s.ranks)))
                 dk[own] = self._reduce_scatter_chunks(dK, sch.chunk_rows[i], s)
@@ -498,13 +747,15 @@ class CPExecutor:
 # --------------------------------------------------------------------------------------------------
 
 class EngineAttention:
-    """attn_fwd / attn_bwd of :class:`CPExecutor` on libzellige: one task handle per schedule (cached),
-    one coalesced forward launch + merge, one backward call.  bf16 CUDA tensors."""
+    """The attention step of :class:`CPExecutor` on libzellige: one task handle per schedule (cached).
+    Pass the bound methods `fwd` / `bwd` for one coalesced forward launch + merge and one backward call after
+    all collectives, or the object itself for launch phases under the collectives.  bf16 CUDA tensors."""
 
-    def __init__(self, head_dim: int, scale: Optional[float] = None, flags: int = 0):
+    def __init__(self, head_dim: int, scale: Optional[float] = None, flags: int = 0, sm_margin: int = 0):
         self.head_dim = head_dim
         self.scale = scale if scale is not None else head_dim ** -0.5
         self.flags = flags
+        self.sm_margin = sm_margin   # SMs left to the communication kernels that run beside a launch phase
         self._handles: Dict[int, object] = {}
 
     def _handle(self, sch: RankSchedule):
@@ -513,8 +764,50 @@ class EngineAttention:
         if h is None:
             h = Z.build_tasks_heads(sch.whole, sch.shards, None, sch.total_q, sch.total_kv, sch.n_heads, self.head_dim,
                                     flags=self.flags)
+            h.set_fwd_phases(sch.fwd_whole_phase, sch.fwd_shard_phase, sch.n_fwd_phases)
+            h.set_bwd_phases(sch.bwd_whole_phase, sch.bwd_shard_phase, sch.n_bwd_phases)
+            if self.sm_margin:
+                h.set_sm_margin(self.sm_margin)
             self._handles[id(sch)] = h
         return h
+
+    # ---- phased form
+    def fwd_begin(self, sch: RankSchedule, Q, K, V):
+        h = self._handle(sch)
+        H, d = sch.n_heads, self.head_dim
+        pr = max(1, int(h.info.partial_rows))
+        return {"h": h, "Q": Q, "K": K, "V": V, "O": torch.zeros_like(Q),
+                "LSE": torch.zeros((H, sch.total_q), dtype=torch.float32, device=Q.device),
+                "OP": torch.empty((pr, H, d), dtype=torch.float32, device=Q.device),
+                "LP": torch.empty((H, pr), dtype=torch.float32, device=Q.device)}
+
+    def fwd_phase(self, sch: RankSchedule, st, phase: int):
+        from . import binding as Z
+        Z.coalesced_attn_fwd_phase(st["h"], phase, st["Q"], st["K"], st["V"], self.scale, st["O"], st["LSE"], st["OP"], st["LP"])
+
+    def fwd_end(self, sch: RankSchedule, st):
+        from . import binding as Z
+        Z.lse_merge(st["h"], st["OP"], st["LP"], st["O"], st["LSE"])
+        return st["O"], (st["Q"], st["K"], st["V"], st["O"], st["LSE"])
+
+    def bwd_begin(self, sch: RankSchedule, saved, dO):
+        h = self._handle(sch)
+        Q, K, V, O, LSE = saved
+        n = int(h.info.bwd_workspace_bytes)
+        return {"h": h, "saved": saved, "dO": dO.contiguous(), "dQ": torch.zeros_like(Q), "dK": torch.zeros_like(K),
+                "dV": torch.zeros_like(V), "ws": torch.empty(n + 256, dtype=torch.uint8, device=Q.device), "n": n}
+
+    def bwd_phase(self, sch: RankSchedule, st, phase: int):
+        from . import binding as Z
+        Q, K, V, O, LSE = st["saved"]
+        Z.coalesced_attn_bwd_phase(st["h"], phase, Q, K, V, O, LSE, st["dO"], self.scale, st["dQ"], st["dK"], st["dV"],
+                                   st["ws"], st["n"])
+
+    def bwd_grads(self, st):
+        return st["dK"], st["dV"]
+
+    def bwd_end(self, sch: RankSchedule, st):
+        return st["dQ"], st["dK"], st["dV"]
 
     def fwd(self, sch: RankSchedule, Q, K, V):
         from . import binding as Z

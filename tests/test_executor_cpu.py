@@ -59,7 +59,76 @@ def _oracle_attention():
     return fwd, bwd
 
 
-def _worker(rank, world, port, out_dir):
+class _PhasedOracle:
+    """The phased attention step on the oracle.  A forward phase evaluates its tasks with the K/V rows as they are
+    at the time of the call (so a task released before its chunk has arrived gives wrong numbers); a backward
+    phase delivers the dK/dV rows of the kv groups of that phase, and dQ with the last one."""
+
+    def __init__(self):
+        sys.path.insert(0, ROOT)
+        from oracle import attention as A
+        self.A, self.scale = A, D ** -0.5
+        self.fwd_calls, self.bwd_calls = [], []
+
+    def fwd_begin(self, sch, Q, K, V):
+        return {"Q": Q, "K": K, "V": V, "whole": {}, "parts": {}}
+
+    def fwd_phase(self, sch, st, phase):
+        A = self.A
+        self.fwd_calls.append(phase)
+        Q, K, V = (st[n].numpy().copy() for n in ("Q", "K", "V"))
+        for w, (off, ln, hb, hc) in enumerate(sch.whole):
+            if sch.fwd_whole_phase[w] != phase:
+                continue
+            st["whole"][w] = {h: A.attn_fwd(np.ascontiguousarray(Q[off:off + ln, h]), np.ascontiguousarray(K[off:off + ln, h]),
+                                            np.ascontiguousarray(V[off:off + ln, h]), self.scale)[0] for h in range(hb, hb + hc)}
+        for si, (qo, ql, ko, kl, _) in enumerate(sch.shards):
+            if sch.fwd_shard_phase[si] != phase:
+                continue
+            st["parts"][si] = [A.attn_fwd(np.ascontiguousarray(Q[qo:qo + ql, h]), np.ascontiguousarray(K[ko:ko + kl, h]),
+                                          np.ascontiguousarray(V[ko:ko + kl, h]), self.scale) for h in range(sch.n_heads)]
+
+    def fwd_end(self, sch, st):
+        A = self.A
+        assert len(st["whole"]) == len(sch.whole) and len(st["parts"]) == len(sch.shards)
+        O = np.zeros(tuple(st["Q"].shape))
+        for w, (off, ln, hb, hc) in enumerate(sch.whole):
+            for h, o in st["whole"][w].items():
+                O[off:off + ln, h] = o
+        groups = {}
+        for si, (qo, ql, _, _, _) in enumerate(sch.shards):
+            groups.setdefault((qo, ql), []).append(si)
+        for (qo, ql), members in groups.items():
+            for h in range(sch.n_heads):
+                O[qo:qo + ql, h] = A.lse_merge([st["parts"][si][h] for si in members])[0]
+        return torch.from_numpy(O), (sch, st["Q"], st["K"], st["V"])
+
+    def bwd_begin(self, sch, saved, dO):
+        import zl_workloads as W
+        _, Q, K, V = saved
+        shards = [tuple(s) + (0, sch.n_heads) for s in sch.shards]
+        p = W.head_range_placement("rank", sch.n_heads, D, 0, sch.whole, shards, sch.total_q, sch.total_kv)
+        g = self.A.placement_bwd(p, Q.numpy(), K.numpy(), V.numpy(), dO.numpy(), scale=self.scale)
+        return {"g": g, "dQ": torch.zeros_like(Q), "dK": torch.zeros_like(K), "dV": torch.zeros_like(V)}
+
+    def bwd_phase(self, sch, st, phase):
+        self.bwd_calls.append(phase)
+        rows = [(off, ln) for w, (off, ln, _, _) in enumerate(sch.whole) if sch.bwd_whole_phase[w] == phase]
+        rows += [(ko, kl) for si, (_, _, ko, kl, _) in enumerate(sch.shards) if sch.bwd_shard_phase[si] == phase]
+        for off, ln in rows:
+            st["dK"][off:off + ln] = torch.from_numpy(st["g"]["dK"][off:off + ln])
+            st["dV"][off:off + ln] = torch.from_numpy(st["g"]["dV"][off:off + ln])
+        if phase == sch.n_bwd_phases - 1:
+            st["dQ"].copy_(torch.from_numpy(st["g"]["dQ"]))
+
+    def bwd_grads(self, st):
+        return st["dK"], st["dV"]
+
+    def bwd_end(self, sch, st):
+        return st["dQ"], st["dK"], st["dV"]
+
+
+def _worker(rank, world, port, out_dir, phased=False):
     sys.path.insert(0, ROOT)
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
@@ -106,10 +175,22 @@ def _worker(rank, world, port, out_dir):
     fwd, bwd = _oracle_attention()
     own = {n: torch.from_numpy(np.concatenate([data[pc.seq_id][t][pc.g0:pc.g1] for pc in sch.pieces]))
            for t, n in enumerate(("q", "k", "v", "do"))}
-    o = ex.forward(own["q"], own["k"], own["v"], fwd)
-    log_f = list(ex.log)
-    dq, dk, dv = ex.backward(own["do"], bwd)
-    log_b = list(ex.log)
+    if phased:
+        step = _PhasedOracle()
+        o = ex.forward(own["q"], own["k"], own["v"], step)
+        log_f = list(ex.log)
+        dq, dk, dv = ex.backward(own["do"], step)
+        log_b = list(ex.log)
+        # every launch phase ran exactly once, the first one before any collective; the backward in order
+        assert sorted(step.fwd_calls) == list(range(sch.n_fwd_phases)) and step.fwd_calls[0] == 0
+        assert step.bwd_calls == list(range(sch.n_bwd_phases))
+        assert sch.n_fwd_phases > 1 and all(ph == 0 for w, ph in enumerate(sch.fwd_whole_phase)
+                                            if segments[[i for i, x in sch.whole_index.items() if x == w][0]].kind == E.WHOLE)
+    else:
+        o = ex.forward(own["q"], own["k"], own["v"], fwd)
+        log_f = list(ex.log)
+        dq, dk, dv = ex.backward(own["do"], bwd)
+        log_b = list(ex.log)
 
     # ---- collectives: decreasing split degree, ties by placement order; the same order on every participant
     degs = [len(e[2]) for e in log_f if e[0] in (E.ALL_GATHER, E.RING, "ulysses_all_to_all")]
@@ -151,6 +232,15 @@ def _worker(rank, world, port, out_dir):
 def test_executor_on_gloo_ranks(tmp_path, world):
     port = 29900 + (os.getpid() * 7 + world) % 300
     mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    assert all(os.path.exists(tmp_path / f"ok{r}") for r in range(world))
+
+
+@pytest.mark.parametrize("world", [2, 4])
+def test_executor_with_launch_phases_on_gloo_ranks(tmp_path, world):
+    """The same layer with the phased attention step: tasks are released as their K/V arrive, the gradients of
+    remote chunks are reduce-scattered after the first backward phase."""
+    port = 29600 + (os.getpid() * 7 + world) % 300
+    mp.spawn(_worker, args=(world, port, str(tmp_path), True), nprocs=world, join=True)
     assert all(os.path.exists(tmp_path / f"ok{r}") for r in range(world))
 
 

@@ -129,3 +129,21 @@ def test_backward_phases_remote_chunks_first(kernel):
     # the plain entry point still does everything in one call
     dQ1, dK1, dV1 = run.backward(Q, K, V, O, LSE, dO)
     assert _same_bits(dK1, dK0) and _same_bits(dV1, dV0)
+
+
+def test_sm_margin_changes_no_result():
+    """Leaving SMs free for communication kernels (zl_set_sm_margin) only changes which CTA runs which item."""
+    p = _placement()
+    Q, K, V, dO = _inputs(p, 6)
+    ref = GpuRun(p)
+    O0, LSE0, _, _ = ref.forward(Q, K, V)
+    dQ0, dK0, dV0 = ref.backward(Q, K, V, O0, LSE0, dO)
+    for margin in (8, 147, 1000):
+        run = GpuRun(p)
+        run.h.set_sm_margin(margin)
+        O, LSE, _, _ = run.forward(Q, K, V)
+        dQ, dK, dV = run.backward(Q, K, V, O, LSE, dO)
+        assert _same_bits(O, O0) and _same_bits(LSE, LSE0) and _same_bits(dK, dK0) and _same_bits(dV, dV0)
+        assert float((dQ.float() - dQ0.float()).norm() / dQ0.float().norm()) <= 1e-4
+    with pytest.raises(run.Z.ZlError):
+        run.h.set_sm_margin(-1)
