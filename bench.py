@@ -299,6 +299,50 @@ def cpu_baseline(p, target_s=12.0):
             "seconds": el}
 
 
+def flash_attn_context(device):
+    """Context only, never the reference arm: the flash_attn package of this image (an mma.sync kernel family built for
+    earlier GPUs) through its varlen call on configuration 2 (whole sequences only: it has no shard tasks), same
+    GPU, same FLOP convention, random bf16 inputs."""
+    import torch
+    import zl_workloads as W
+    try:
+        from flash_attn import flash_attn_varlen_func
+        p = W.config(2)
+        H, d, T = p.n_heads, p.head_dim, p.total_q
+        q, k, v = (torch.randn(T, H, d, device=device, dtype=torch.bfloat16, requires_grad=True) for _ in range(3))
+        do = torch.randn(T, H, d, device=device, dtype=torch.bfloat16)
+        cu = torch.tensor(p.cu_seqlens, dtype=torch.int32, device=device)
+        mx = max(b - a for a, b in zip(p.cu_seqlens[:-1], p.cu_seqlens[1:]))
+
+        def fwd():
+            return flash_attn_varlen_func(q, k, v, cu, cu, mx, mx, softmax_scale=d ** -0.5, causal=False)
+
+        def step():
+            fwd().backward(do)
+            q.grad = k.grad = v.grad = None
+
+        def timed(fn, n=10):
+            for _ in range(3):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(n):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / n
+
+        ms_step = timed(step)
+        with torch.no_grad():
+            ms_fwd = timed(fwd)
+        return {"what": "flash_attn varlen (library, mma.sync) on cfg2_images, same GPU", "fwd_ms": ms_fwd,
+                "fwd_tflops": p.fwd_flops() / ms_fwd / 1e9, "fwd_bwd_ms": ms_step,
+                "fwd_bwd_tflops": (p.fwd_flops() + p.bwd_flops()) / ms_step / 1e9}
+    except Exception as e:  # noqa: BLE001  (package missing or not runnable on this GPU)
+        return {"what": "flash_attn varlen on cfg2_images", "unavailable": repr(e)[:200]}
+
+
 def run_ours(args):
     import torch
     import zl_workloads as W
@@ -411,6 +455,10 @@ def run_ours(args):
                    "parallelism": f"{world} independent rank-local placements"},
         "fwd_tflops": aggregate_tflops(world, p.fwd_flops(), ms_fwd / K),
         "fwd_ms": ms_fwd / K,
+        # with activation checkpointing (the paper's training setting, Section V-A) a layer costs two forwards and one
+        # backward; the forward is counted twice in both the time and the FLOPs
+        "step_equivalent": {"what": "2 x fwd + bwd (recompute)", "ms": ms_step + ms_fwd / K,
+                            "tflops": aggregate_tflops(world, 2 * p.fwd_flops() + p.bwd_flops(), ms_step + ms_fwd / K)},
         # the datasheet dense BF16 figure first: that is the peak the metric names (its 60 % mark is 1350 TFLOP/s)
         "frac_of_peak": {"datasheet_2250": value / world / 2250.0,
                          "measured_burst": value / world / float(peaks.get("bf16_tflops", 1590.0)),
@@ -423,6 +471,8 @@ def run_ours(args):
         "clocks": clocks,
     }
 
+    if world == 1 and args.context_flash_attn:
+        result["context"] = flash_attn_context(device)
     if world == 1 and args.extra_configs:
         extra = {}
         del wl
@@ -646,6 +696,8 @@ def main():
     ap.add_argument("--cp", action="store_true",
                     help="context-parallel mode: one video under N-way all-gather CP across the N ranks + images per rank, "
                          "through the executor (printed as its own JSON line, not the headline)")
+    ap.add_argument("--context-flash-attn", action="store_true",
+                    help="also time the image's flash_attn package on configuration 2 (context line, N=1)")
     ap.add_argument("--bwd-kernel", type=int, default=0, choices=[0, 1, 2],
                     help="backward main kernel: 0 library default, 1 one CTA per key tile, 2 CTA pairs")
     ap.add_argument("--ablation", default="", choices=["", "straggler", "coalescing"],
