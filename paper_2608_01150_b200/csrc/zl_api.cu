@@ -526,8 +526,10 @@ zl_status bwd_impl(const zl_tasks* t, int32_t phase, const void* q, const void* 
     }
     const bool pair = s.head_dim == 128 && (t->bwd_kernel == 2 || (t->bwd_kernel == 0 && kDefaultBwdPair));
     if (p.n_items > 0 && pair) {
-        CUtensorMap tq64, tdo64, taug, tdq16;
+        CUtensorMap tq64, tdo64, taug, tdq16, tdk32, tdv32;
         if (!make_tmap_f32_acc(&tdq16, ws + s.ws_dq_acc_off, s.q_pad_total, s.n_heads, s.head_dim, 32, 16) ||
+            !make_tmap(&tdk32, dk, s.total_kv, s.n_heads, s.head_dim, 32, grad_stride) ||
+            !make_tmap(&tdv32, dv, s.total_kv, s.n_heads, s.head_dim, 32, grad_stride) ||
             !make_tmap(&tq64, q, s.total_q, s.n_heads, s.head_dim, 64, in_stride) ||
             !make_tmap(&tdo64, d_o, s.total_q, s.n_heads, s.head_dim, 64, hd) ||
             !make_tmap_aug_rows(&taug, p.aug, (s.q_pad_total / kTileQ) * s.n_heads))
@@ -539,7 +541,7 @@ zl_status bwd_impl(const zl_tasks* t, int32_t phase, const void* q, const void* 
         pp.n_items = pi1 - pi0;
         const int n_clusters = std::min<int>(std::max(2, t->n_sms - t->sm_margin) / 2, pp.n_items);
         LaunchTimer lt(t, ZL_K_BWD_MAIN, cs);
-        if (launch_bwd_pair(tq, tq64, tk, tv, tdo, tdo64, tdq16, taug, pp, n_clusters, cs) != cudaSuccess) return ZL_ERR_CUDA;
+        if (launch_bwd_pair(tq, tq64, tk, tv, tdo, tdo64, tdq16, taug, tdk32, tdv32, pp, n_clusters, cs) != cudaSuccess) return ZL_ERR_CUDA;
         g_launches.fetch_add(1);
     } else if (p.n_items > 0) {
         const int grid = std::min<int>(std::max(2, t->n_sms - t->sm_margin), p.n_items);

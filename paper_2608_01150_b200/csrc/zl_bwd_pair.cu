@@ -147,6 +147,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_do64,
                    const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_aug,
+                   const __grid_constant__ CUtensorMap tm_dk32, const __grid_constant__ CUtensorMap tm_dv32,
                    const BwdParams p) {
     using Smem = PairSmem;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -459,6 +460,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t dst_full_l = map_to_cta(smem_u32(&sm.dst_full), 0);
         const float sl2 = p.scale_log2;
         uint32_t item_cnt = 0, it_cnt = 0;
+        bool store_pending = false;  // warp-uniform
         #pragma unroll 1
         for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
             const WorkItem wi = p.items[it];
@@ -544,6 +546,11 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         // (same swizzle: the box is copied to the same offset modulo 1024 in the partner), once the
                         // dQ MMAs of the previous tile have consumed the boxes in both CTAs
                         if (it_cnt > 0) ZL_WAIT_WARP(&sm.ds_free, (it_cnt - 1) & 1, 33);
+                        if (store_pending) {  // the previous item's last gradient store still reads this warp's box
+                            if (lane == 0) bulk_wait_group_read<0>();
+                            __syncwarp();
+                            store_pending = false;
+                        }
 #pragma unroll
                         for (int c16 = 0; c16 < 8; ++c16)
                             st_shared_v4(ds_row_dst + ((c16 ^ (row & 7)) << 4), dd[c16 * 4], dd[c16 * 4 + 1], dd[c16 * 4 + 2],
@@ -565,21 +572,63 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const float sc = (wg == 0) ? 1.f : p.scale;
             const uint32_t col_acc = (wg == 0) ? kColDV : kColDK;
             const int64_t grow = (int64_t)g.kv_off + wi.row0 + kTileKV * (int)rank + row;
-            __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + grow * p.grad_row_stride + wi.head * D;
+            if (quarter * 32 + 32 <= rows_here) {
+                // all 32 rows of this warp are inside the item: stage 64 columns at a time in the 4 KB of the dS
+                // operand that only this warp writes (its rows of the in-place box, or its outgoing box) and
+                // write each with one TMA store -- coalesced, and the warp moves on while the copy engine drains
+                // the box.  The last dQ MMAs read that box and are not covered by acc_full (another thread
+                // issued them): wait for them here, as the next hand-over would.
+                ZL_WAIT_WARP(&sm.ds_free, (it_cnt - 1) & 1, 42);
+                const uint32_t box = ds_local ? smem_u32(sm.ds[rank]) + quarter * 4096 : smem_u32(sm.ds_out[quarter]);
+                const uint32_t box_row = box + lane * 128;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_x32(lane_addr + col_acc + c * 32, r);
-                tmem_wait_ld();
-                if (row_ok) {
+                for (int b = 0; b < 2; ++b) {
+                    if (b > 0) {
+                        if (lane == 0) bulk_wait_group_read<0>();
+                        __syncwarp();
+                    }
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 o4;
-                        o4.x = pack_bf16(__uint_as_float(r[i]) * sc, __uint_as_float(r[i + 1]) * sc);
-                        o4.y = pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc);
-                        o4.z = pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc);
-                        o4.w = pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc);
-                        *reinterpret_cast<uint4*>(dst + c * 32 + i) = o4;
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_x32(lane_addr + col_acc + b * 64 + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            const int i = k4 * 8;
+                            st_shared_v4(box_row + (((c * 4 + k4) ^ (lane & 7)) << 4),
+                                         pack_bf16(__uint_as_float(r[i]) * sc, __uint_as_float(r[i + 1]) * sc),
+                                         pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc),
+                                         pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc),
+                                         pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc));
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                                     ::"l"(reinterpret_cast<uint64_t>(wg == 0 ? &tm_dv32 : &tm_dk32)), "r"(box), "r"(b * 64),
+                                       "r"(wi.head), "r"((int)(grow - lane)) : "memory");
+                        bulk_commit_group();
+                    }
+                }
+                store_pending = true;
+            } else {
+                __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + grow * p.grad_row_stride + wi.head * D;
+#pragma unroll 1
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_x32(lane_addr + col_acc + c * 32, r);
+                    tmem_wait_ld();
+                    if (row_ok) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8) {
+                            uint4 o4;
+                            o4.x = pack_bf16(__uint_as_float(r[i]) * sc, __uint_as_float(r[i + 1]) * sc);
+                            o4.y = pack_bf16(__uint_as_float(r[i + 2]) * sc, __uint_as_float(r[i + 3]) * sc);
+                            o4.z = pack_bf16(__uint_as_float(r[i + 4]) * sc, __uint_as_float(r[i + 5]) * sc);
+                            o4.w = pack_bf16(__uint_as_float(r[i + 6]) * sc, __uint_as_float(r[i + 7]) * sc);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + i) = o4;
+                        }
                     }
                 }
             }
@@ -665,7 +714,8 @@ teardown:
 
 cudaError_t launch_bwd_pair(const CUtensorMap& tq, const CUtensorMap& tq64, const CUtensorMap& tk, const CUtensorMap& tv,
                             const CUtensorMap& tdo, const CUtensorMap& tdo64, const CUtensorMap& tdq,
-                            const CUtensorMap& taug, const BwdParams& p, int n_clusters, cudaStream_t stream) {
+                            const CUtensorMap& taug, const CUtensorMap& tdk32, const CUtensorMap& tdv32, const BwdParams& p,
+                            int n_clusters, cudaStream_t stream) {
     if (p.n_items == 0) return cudaSuccess;
     constexpr int smem = sizeof(PairSmem);
     constexpr int kMaxDevices = 64;
@@ -678,7 +728,7 @@ cudaError_t launch_bwd_pair(const CUtensorMap& tq, const CUtensorMap& tq64, cons
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
     }
-    zl_bwd_pair_kernel<<<2 * n_clusters, kPairThreads, smem, stream>>>(tq, tq64, tk, tv, tdo, tdo64, tdq, taug, p);
+    zl_bwd_pair_kernel<<<2 * n_clusters, kPairThreads, smem, stream>>>(tq, tq64, tk, tv, tdo, tdo64, tdq, taug, tdk32, tdv32, p);
     return cudaGetLastError();
 }
 

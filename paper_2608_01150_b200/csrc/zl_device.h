@@ -68,10 +68,12 @@ cudaError_t launch_bwd_main(int head_dim, const CUtensorMap& tq, const CUtensorM
                             const CUtensorMap& tdo, const CUtensorMap& tdq, const CUtensorMap& tdk,
                             const CUtensorMap& tdv, const BwdParams& p, int grid, cudaStream_t stream);
 // CTA-pair form of the main kernel (head_dim 128): `p.items` is the pair item list, `tq64` / `tdo64` are maps
-// with 64-row boxes, `taug` views the augmentation tiles as rows of 1 KB.
+// with 64-row boxes, `taug` views the augmentation tiles as rows of 1 KB, `tdk32` / `tdv32` are the gradient maps
+// with 32-row boxes (one warp's rows).
 cudaError_t launch_bwd_pair(const CUtensorMap& tq, const CUtensorMap& tq64, const CUtensorMap& tk, const CUtensorMap& tv,
                             const CUtensorMap& tdo, const CUtensorMap& tdo64, const CUtensorMap& tdq,
-                            const CUtensorMap& taug, const BwdParams& p, int n_clusters, cudaStream_t stream);
+                            const CUtensorMap& taug, const CUtensorMap& tdk32, const CUtensorMap& tdv32, const BwdParams& p,
+                            int n_clusters, cudaStream_t stream);
 cudaError_t launch_bwd_post(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream);
 
 cudaError_t launch_fwd(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
