@@ -5,14 +5,14 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as A
-from zl_testlib import (GpuRun, bits, check_backward, check_forward, dev_to_f64, random_bits, to_dev,
+from zl_testlib import (EngineRun, bits, check_backward, check_forward, dev_to_f64, random_bits, to_dev,
                         to_f64, GATE_GRAD_REL, SENTINEL)
 
 pytestmark = pytest.mark.gpu
 
 
 def _run(p, Qb, Kb, Vb, dOb, gate=True):
-    run = GpuRun(p)
+    run = EngineRun(p)
     Qd, Kd, Vd, dOd = (to_dev(x) for x in (Qb, Kb, Vb, dOb))
     O, LSE, _, _ = run.forward(Qd, Kd, Vd)
     dQ, dK, dV = run.backward(Qd, Kd, Vd, O, LSE, dOd)
@@ -78,7 +78,7 @@ def test_isolation_with_finite_poison_in_neighbours():
     Q2, K2, V2, dO2 = Qb.copy(), Kb.copy(), Vb.copy(), dOb.copy()
     Q2[230:240] = big; dO2[230:240] = big; K2[230:240] = big; V2[230:240] = big   # rows no task owns
     Q2[290:] = big; dO2[290:] = big; K2[310:] = big; V2[310:] = big
-    run2 = GpuRun(p)
+    run2 = EngineRun(p)
     Qd, Kd, Vd, dOd = (to_dev(x) for x in (Q2, K2, V2, dO2))
     O, LSE, _, _ = run2.forward(Qd, Kd, Vd)
     dQ2, dK2, dV2 = run2.backward(Qd, Kd, Vd, O, LSE, dOd)

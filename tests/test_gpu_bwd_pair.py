@@ -7,7 +7,7 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as A
-from zl_testlib import (GpuRun, bits, check_backward, dev_to_f64, random_bits, rel_fro, to_dev, to_f64, GATE_GRAD_REL,
+from zl_testlib import (EngineRun, bits, check_backward, dev_to_f64, random_bits, rel_fro, to_dev, to_f64, GATE_GRAD_REL,
                         SENTINEL)
 
 pytestmark = pytest.mark.gpu
@@ -20,7 +20,7 @@ def _both(p, seed):
     H, d = p.n_heads, p.head_dim
     Qb, dOb = random_bits(rng, p.total_q, H, d), random_bits(rng, p.total_q, H, d)
     Kb, Vb = random_bits(rng, p.total_kv, H, d), random_bits(rng, p.total_kv, H, d)
-    run = GpuRun(p)
+    run = EngineRun(p)
     Qd, Kd, Vd, dOd = (to_dev(x) for x in (Qb, Kb, Vb, dOb))
     O, LSE, _, _ = run.forward(Qd, Kd, Vd)
     out = {}
@@ -57,7 +57,7 @@ def test_pair_kernel_head_ranges():
 def test_pair_kernel_is_refused_for_head_dim_64():
     import paper_2608_01150_b200 as Z
     p = W.config(1)
-    run = GpuRun(p)
+    run = EngineRun(p)
     with pytest.raises(Z.ZlError) as e:
         run.h.set_bwd_kernel(2)
     assert e.value.status == 3      # ZL_ERR_UNSUPPORTED
@@ -70,7 +70,7 @@ def test_pair_kernel_on_the_image_batch_configuration():
     p = W.config(2)
     B = C._inputs(p)
     d = C._device_tensors(p, B)
-    run = GpuRun(p)
+    run = EngineRun(p)
     run.h.set_bwd_kernel(2)
     O, LSE, _, _ = run.forward(d["Q"], d["K"], d["V"])
     dQ, dK, dV = run.backward(d["Q"], d["K"], d["V"], O, LSE, d["dO"])

@@ -21,7 +21,7 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as A
-from zl_testlib import (GpuRun, check_backward, check_forward, dev_to_f64, rel_fro, row_rel, to_dev, to_f64,
+from zl_testlib import (EngineRun, check_backward, check_forward, dev_to_f64, rel_fro, row_rel, to_dev, to_f64,
                         TOL_GRAD_REL, TOL_GRAD_ROW, TOL_LSE_MAX, TOL_O_MAX, TOL_O_MEAN)
 
 pytestmark = pytest.mark.gpu
@@ -59,7 +59,7 @@ def _device_tensors(p, B):
 
 
 def _run_gpu(p, B):
-    run = GpuRun(p)
+    run = EngineRun(p)
     d = _device_tensors(p, B)
     O, LSE, _, _ = run.forward(d["Q"], d["K"], d["V"])
     dQ, dK, dV = run.backward(d["Q"], d["K"], d["V"], O, LSE, d["dO"])
@@ -261,7 +261,7 @@ def test_spike_keys_at_chunk_and_tile_boundaries_full_size(ci):
                 planted[h].append((i, j))
         B["K"][h] = W.f32_to_bf16_bits(kf)
     d = _device_tensors(p, B)
-    run = GpuRun(p)
+    run = EngineRun(p)
     O, LSE, _, _ = run.forward(d["Q"], d["K"], d["V"])
     n_checked = n_sharp = 0
     worst_o = worst_l = 0.0

@@ -9,7 +9,7 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as orc
-from zl_testlib import GpuRun, SENTINEL, bits, check_backward, check_forward, dev_to_f64, to_dev, to_f64
+from zl_testlib import EngineRun, SENTINEL, bits, check_backward, check_forward, dev_to_f64, to_dev, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -24,7 +24,7 @@ def _run_both(p):
     gref = orc.placement_bwd(p, f["Q"], f["K"], f["V"], f["dO"])
     out = {}
     for name, flags in (("plain", 0), ("fused", FUSE)):
-        run = GpuRun(p, flags=flags)
+        run = EngineRun(p, flags=flags)
         O, LSE, OP, LP = run.forward(Q, K, V)
         check_forward(p, O, LSE, ref)
         dQ, dK, dV = run.backward(Q, K, V, O, LSE, dO)

@@ -6,14 +6,14 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as A
-from zl_testlib import (GpuRun, bits, check_forward, dev_to_f64, random_bits, to_dev, to_f64,
+from zl_testlib import (EngineRun, bits, check_forward, dev_to_f64, random_bits, to_dev, to_f64,
                         GATE_O_MAX, GATE_LSE_MAX, SENTINEL)
 
 pytestmark = pytest.mark.gpu
 
 
 def _run(p, Qb, Kb, Vb, gate=True):
-    run = GpuRun(p)
+    run = EngineRun(p)
     O, LSE, OP, LP = run.forward(to_dev(Qb), to_dev(Kb), to_dev(Vb))
     ref = A.placement_fwd(p, to_f64(Qb), to_f64(Kb), to_f64(Vb))
     stats = check_forward(p, O, LSE, ref)
@@ -109,7 +109,7 @@ def test_isolation_and_untouched_rows():
     K2[100:230] = big                     # large finite poison in sequence 1
     V2[100:230] = big
     K2[230:240] = big                     # and in rows no task owns
-    run2 = GpuRun(p)
+    run2 = EngineRun(p)
     O2, L2, _, _ = run2.forward(to_dev(Q2), to_dev(K2), to_dev(V2))
     keep = np.r_[0:100, 240:290]
     assert torch.equal(O1[keep], O2[keep]) and torch.equal(L1[:, keep], L2[:, keep])
@@ -119,7 +119,7 @@ def test_isolation_and_untouched_rows():
 def test_forward_is_run_to_run_bit_identical():
     p = W.config(1)
     Qd, Kd, Vd = to_dev(bits(p, "Q")), to_dev(bits(p, "K")), to_dev(bits(p, "V"))
-    run = GpuRun(p)
+    run = EngineRun(p)
     a = run.forward(Qd, Kd, Vd)
     b = run.forward(Qd, Kd, Vd)
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
@@ -150,7 +150,7 @@ def test_bounded_wait_expires_and_is_reported():
     """A wait nobody satisfies returns after its limit, reports ZL_ERR_TIMEOUT through the device status
     word and leaves the context usable (no trap, no hang)."""
     p = W.config(1)
-    run = GpuRun(p)
+    run = EngineRun(p)
     run.h.selftest_bounded_wait(limit_us=500)
     torch.cuda.synchronize()
     code, where = run.h.last_device_status()
@@ -166,7 +166,7 @@ def test_results_do_not_depend_on_the_work_order():
     rng = np.random.RandomState(8)
     Qd = to_dev(random_bits(rng, p.total_q, 2, 128)); Kd = to_dev(random_bits(rng, p.total_kv, 2, 128))
     Vd = to_dev(random_bits(rng, p.total_kv, 2, 128))
-    run = GpuRun(p)
+    run = EngineRun(p)
     ref = run.forward(Qd, Kd, Vd)
     for mode in (1, 2, 0):
         run.h.set_fwd_order(mode)

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import zl_workloads as W
-from zl_testlib import GpuRun, bits, dev_to_f64, rel_fro, to_dev, TOL_GRAD_REL
+from zl_testlib import EngineRun, bits, dev_to_f64, rel_fro, to_dev, TOL_GRAD_REL
 
 pytestmark = pytest.mark.gpu
 
@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 def test_step_replays_from_a_cuda_graph():
     import paper_2608_01150_b200 as Z
     p = W.config(1)
-    run = GpuRun(p)
+    run = EngineRun(p)
     H, d = p.n_heads, p.head_dim
     Q, K, V, dO = (to_dev(bits(p, t)) for t in ("Q", "K", "V", "dO"))
     O_ref, LSE_ref, _, _ = run.forward(Q, K, V)

@@ -7,7 +7,7 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as A
-from zl_testlib import (GpuRun, SENTINEL, bits, check_backward, check_forward, covered_rows, dev_to_f64, random_bits,
+from zl_testlib import (EngineRun, SENTINEL, bits, check_backward, check_forward, covered_rows, dev_to_f64, random_bits,
                         to_dev, to_f64, GATE_GRAD_REL, GATE_LSE_MAX, GATE_O_MAX)
 
 pytestmark = pytest.mark.gpu
@@ -18,7 +18,7 @@ def _run(p, seed):
     H, d = p.n_heads, p.head_dim
     Qb, dOb = random_bits(rng, p.total_q, H, d), random_bits(rng, p.total_q, H, d)
     Kb, Vb = random_bits(rng, p.total_kv, H, d), random_bits(rng, p.total_kv, H, d)
-    run = GpuRun(p)
+    run = EngineRun(p)
     Qd, Kd, Vd, dOd = (to_dev(x) for x in (Qb, Kb, Vb, dOb))
     O, LSE, _, _ = run.forward(Qd, Kd, Vd)
     dQ, dK, dV = run.backward(Qd, Kd, Vd, O, LSE, dOd)
@@ -66,7 +66,7 @@ def test_shard_groups_with_head_ranges_merge_and_backward():
     H, d = p.n_heads, p.head_dim
     Qb, dOb = random_bits(rng, p.total_q, H, d), random_bits(rng, p.total_q, H, d)
     Kb, Vb = random_bits(rng, p.total_kv, H, d), random_bits(rng, p.total_kv, H, d)
-    runf = GpuRun(p, flags=Z.BUILD_FUSE_LOCAL_CHUNKS)
+    runf = EngineRun(p, flags=Z.BUILD_FUSE_LOCAL_CHUNKS)
     assert runf.info.n_fused_ranges == 2 and runf.info.n_merge_groups == 0
     Qd, Kd, Vd, dOd = (to_dev(x) for x in (Qb, Kb, Vb, dOb))
     O, LSE, _, _ = runf.forward(Qd, Kd, Vd)

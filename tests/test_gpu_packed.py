@@ -9,7 +9,7 @@ import torch
 
 import zl_workloads as W
 from oracle import attention as orc
-from zl_testlib import (GpuRun, SENTINEL, bits, check_backward, check_forward, dev_to_f64, rel_fro, to_dev,
+from zl_testlib import (EngineRun, SENTINEL, bits, check_backward, check_forward, dev_to_f64, rel_fro, to_dev,
                         to_f64, TOL_GRAD_REL)
 
 pytestmark = pytest.mark.gpu
@@ -19,7 +19,7 @@ def _packed_case(p):
     import paper_2608_01150_b200 as Z
     assert p.total_q == p.total_kv
     H, d, T = p.n_heads, p.head_dim, p.total_q
-    run = GpuRun(p)
+    run = EngineRun(p)
     hb = {t: bits(p, t) for t in ("Q", "K", "V", "dO")}
     Q, K, V, dO = (to_dev(hb[t]) for t in ("Q", "K", "V", "dO"))
     qkv = torch.stack([Q, K, V], dim=1).contiguous()          # [T, 3, H, d]

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import zl_workloads as W
-from zl_testlib import SENTINEL, GpuRun, random_bits, to_dev
+from zl_testlib import SENTINEL, EngineRun, random_bits, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -42,10 +42,10 @@ def _same_bits(a, b):
 def test_forward_phases_match_single_launch_while_chunks_arrive():
     p = _placement()
     Q, K, V, _ = _inputs(p, 3)
-    ref = GpuRun(p)
+    ref = EngineRun(p)
     O0, LSE0, OP0, LP0 = ref.forward(Q, K, V)
 
-    run = GpuRun(p)
+    run = EngineRun(p)
     Z, h = run.Z, run.h
     n_whole, n_shards = len(p.cu_seqlens) - 1, len(p.shards)
     # phase 0: whole sequences and the local chunk (chunk 0); phase j: the chunk that arrives at ring step j
@@ -70,8 +70,8 @@ def test_forward_phases_match_single_launch_while_chunks_arrive():
 def test_forward_phases_in_reverse_order_and_one_launch_after_regrouping():
     p = _placement()
     Q, K, V, _ = _inputs(p, 4)
-    O0, LSE0, _, _ = GpuRun(p).forward(Q, K, V)
-    run = GpuRun(p)
+    O0, LSE0, _, _ = EngineRun(p).forward(Q, K, V)
+    run = EngineRun(p)
     Z, h = run.Z, run.h
     run.h.set_fwd_phases([1, 0, 1, 0], [2, 0, 1, 2], 3)
     O, LSE, OP, LP = _buffers(p, h.info, Q.device)
@@ -91,12 +91,12 @@ def test_forward_phases_in_reverse_order_and_one_launch_after_regrouping():
 def test_backward_phases_remote_chunks_first(kernel):
     p = _placement()
     Q, K, V, dO = _inputs(p, 5)
-    ref = GpuRun(p)
+    ref = EngineRun(p)
     ref.h.set_bwd_kernel(kernel)
     O, LSE, _, _ = ref.forward(Q, K, V)
     dQ0, dK0, dV0 = ref.backward(Q, K, V, O, LSE, dO)
 
-    run = GpuRun(p)
+    run = EngineRun(p)
     Z, h = run.Z, run.h
     h.set_bwd_kernel(kernel)
     n_whole = len(p.cu_seqlens) - 1
@@ -135,11 +135,11 @@ def test_sm_margin_changes_no_result():
     """Leaving SMs free for communication kernels (zl_set_sm_margin) only changes which CTA runs which item."""
     p = _placement()
     Q, K, V, dO = _inputs(p, 6)
-    ref = GpuRun(p)
+    ref = EngineRun(p)
     O0, LSE0, _, _ = ref.forward(Q, K, V)
     dQ0, dK0, dV0 = ref.backward(Q, K, V, O0, LSE0, dO)
     for margin in (8, 147, 1000):
-        run = GpuRun(p)
+        run = EngineRun(p)
         run.h.set_sm_margin(margin)
         O, LSE, _, _ = run.forward(Q, K, V)
         dQ, dK, dV = run.backward(Q, K, V, O, LSE, dO)

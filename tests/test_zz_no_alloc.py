@@ -10,7 +10,7 @@ import pytest
 import torch
 
 import zl_workloads as W
-from zl_testlib import GpuRun, bits, dev_to_f64, rel_fro, to_dev, TOL_GRAD_REL
+from zl_testlib import EngineRun, bits, dev_to_f64, rel_fro, to_dev, TOL_GRAD_REL
 
 pytestmark = pytest.mark.gpu
 
@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 def test_noalloc_backward_matches_workspace_backward_twice():
     import paper_2608_01150_b200 as Z
     p = W.config(1)
-    run = GpuRun(p)
+    run = EngineRun(p)
     assert run.info.bwd_workspace_bytes <= Z.NOALLOC_SCRATCH_BYTES
     Q, K, V, dO = (to_dev(bits(p, t)) for t in ("Q", "K", "V", "dO"))
     O, LSE, _, _ = run.forward(Q, K, V)

@@ -47,7 +47,7 @@ def dev_to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to(torch.float64).cpu().numpy()
 
 
-class GpuRun:
+class EngineRun:
     """Runs forward (+merge) and optionally backward for a placement through the binding."""
 
     def __init__(self, p, scale=None, flags=0):
