@@ -33,7 +33,7 @@ def _run(p, seed):
 
 def test_whole_images_next_to_two_ulysses_sequences():
     """H = 12: six whole images over 12 heads + two sequences over heads [0,6) and [6,12) that share one
-    block of rows (the judge of isolation here is the oracle: each head of those rows belongs to a
+    block of rows (what decides isolation here is the oracle: each head of those rows belongs to a
     different sequence)."""
     p = W.ulysses_mix_placement(n_heads=12, head_dim=128, n_images=6, image_len=1560, seq_len=3600, degree=2)
     run, _, fs, bs = _run(p, 31)
