@@ -388,9 +388,10 @@ def run_ours(args):
     kt = wl.h.get_kernel_timing()
     wl.h.set_kernel_timing(False)
     tot = sum(v[0] for v in kt.values()) or 1.0
-    kernels = {k: {"launches": v[1], "avg_ms": (v[0] / v[1] if v[1] else None), "share": v[0] / tot}
+    kernels = {k: {"launches": v[1], "avg_ms": (v[0] / v[1] if v[1] else None), "ms_per_step": v[0] / K, "share": v[0] / tot}
                for k, v in kt.items()}
-    bm = kernels["bwd_main"]["avg_ms"]
+    # per step, not per launch: a placement with many short sequences runs its last key tiles in a second launch
+    bm = kernels["bwd_main"]["ms_per_step"] or None
     peak_t = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     achieved = p.bwd_flops() / (bm * 1e-3) / 1e12 if bm else None
     pair = p.head_dim == 128 and args.bwd_kernel != 1   # the library's default at head_dim 128 is the CTA-pair kernel
@@ -422,9 +423,9 @@ def run_ours(args):
         roofline["smem"] = {"bytes_per_tile_pair": per_pair, "tile_pairs": n_pairs, "achieved": b_clk, "peak": 128.0,
                             "unit": "B/clk/SM", "frac": b_clk / 128.0,
                             "note": "shared-memory traffic of the same launches over the sampled median SM clock"}
-    fm = kernels["fwd"]["avg_ms"]
+    fm = kernels["fwd"]["ms_per_step"] or None
     fwd_kernel_tflops = p.fwd_flops() / (fm * 1e-3) / 1e12 if fm else None
-    mm = kernels["merge"]["avg_ms"]
+    mm = kernels["merge"]["ms_per_step"] or None
     merge_gbs = wl.merge_bytes / (mm * 1e-3) / 1e9 if mm else None
 
     # end to end with host buffers
