@@ -38,7 +38,7 @@ METRIC = "coalesced attention TFLOP/s fwd and fwd+bwd; % of B200 dense BF16 peak
 # DRAM traffic of one launch of the backward main kernel (dram__bytes_read.sum + dram__bytes_write.sum, a one-pass
 # ncu capture; profiles/zl_bwd_pair_kernel_cfg4_dram.txt), keyed by (configuration, kernel).  It is reported only for
 # the workload and kernel it was measured on; any other combination reports null.
-NCU_BWD_DRAM_BYTES = {(4, "zl_bwd_pair_kernel"): 8.51e9 + 5.00e9,
+NCU_BWD_DRAM_BYTES = {(4, "zl_bwd_pair_kernel"): 9.32e9 + 5.42e9,
                       (3, "zl_bwd_pair_kernel"): 2.384398592e9 + 1.395509248e9,
                       (3, "zl_bwd_main_kernel"): 2.647806e9 + 1.529451e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
