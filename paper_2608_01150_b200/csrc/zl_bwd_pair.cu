@@ -581,13 +581,13 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ZL_WAIT_WARP(&sm.ds_free, (it_cnt - 1) & 1, 42);
                 const uint32_t box = ds_local ? smem_u32(sm.ds[rank]) + quarter * 4096 : smem_u32(sm.ds_out[quarter]);
                 const uint32_t box_row = box + lane * 128;
-#pragma unroll
+#pragma unroll 1
                 for (int b = 0; b < 2; ++b) {
                     if (b > 0) {
                         if (lane == 0) bulk_wait_group_read<0>();
                         __syncwarp();
                     }
-#pragma unroll
+#pragma unroll 1
                     for (int c = 0; c < 2; ++c) {
                         uint32_t r[32];
                         tmem_ld_x32(lane_addr + col_acc + b * 64 + c * 32, r);
