@@ -722,7 +722,7 @@ cudaError_t launch_main_t(const CUtensorMap& tq, const CUtensorMap& tk, const CU
 
 cudaError_t launch_bwd_pre(int head_dim, const BwdParams& p, int n_sms, cudaStream_t stream) {
     if (p.q_pad_total == 0) return cudaSuccess;
-    const int grid = n_sms * 8;
+    const int grid = n_sms * 2;  // what is resident at once (two units per warp in flight need 92 registers): no block waves
     if (head_dim == 128) zl_bwd_pre_kernel<128><<<grid, kPreThreads, 0, stream>>>(p);
     else zl_bwd_pre_kernel<64><<<grid, kPreThreads, 0, stream>>>(p);
     return cudaGetLastError();
