@@ -64,7 +64,9 @@ struct PairSmem {
     alignas(1024) uint8_t aug_s[2048];              // [pieces of -LSE/scale of this CTA's 64 queries | zeros]
     alignas(1024) uint8_t aug_d[2048];              // [pieces of -D | zeros]
     alignas(1024) uint8_t ones[2][2048];            // [ones in elements 0..2][zeros]
-    alignas(8) uint64_t kv_full, kv_empty, kx_empty;
+    // K, V and the K columns for dQ are filled and released separately: K is free after the item's last S^T, V after
+    // its last dP^T, the K columns after its last dQ, and the next item's tiles are loaded as soon as each one is
+    alignas(8) uint64_t k_full, k_empty, v_full, v_empty, kx_full, kx_empty;
     uint64_t qr_full, qr_empty, qc_full, qc_empty;
     uint64_t dor_full, dor_empty, doc_full, doc_empty;  // dO rows + D pieces (B of dP^T) and dO columns (B of dV) have different lifetimes
     uint64_t s_full, dp_full, p_full, dst_full, ds_full, ds_free, dq_full, acc_full;
@@ -168,8 +170,11 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         return;
     }
     if (threadIdx.x == 0) {
-        mbar_init(&sm.kv_full, 1);
-        mbar_init(&sm.kv_empty, 1);
+        mbar_init(&sm.k_full, 1);
+        mbar_init(&sm.k_empty, 1);
+        mbar_init(&sm.v_full, 1);
+        mbar_init(&sm.v_empty, 1);
+        mbar_init(&sm.kx_full, 1);
         mbar_init(&sm.kx_empty, 1);
         mbar_init(&sm.qr_full, 1);
         mbar_init(&sm.qr_empty, 1);
@@ -233,7 +238,8 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // -------------------------------------------------------------- TMA producer: K, V, Q rows, dO
             // Transaction bytes of both CTAs are counted on the leader's barrier, which the leader's
             // producer arms for the pair.
-            const uint32_t kv_full_l = map_to_cta(smem_u32(&sm.kv_full), 0);
+            const uint32_t k_full_l = map_to_cta(smem_u32(&sm.k_full), 0);
+            const uint32_t v_full_l = map_to_cta(smem_u32(&sm.v_full), 0);
             const uint32_t qr_full_l = map_to_cta(smem_u32(&sm.qr_full), 0);
             const uint32_t dor_full_l = map_to_cta(smem_u32(&sm.dor_full), 0);
             const uint32_t doc_full_l = map_to_cta(smem_u32(&sm.doc_full), 0);
@@ -243,14 +249,14 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
                 const int key0 = g.kv_off + wi.row0;   // first key row of the pair
-                ZL_WAIT(&sm.kv_empty, (item_cnt & 1) ^ 1, 1);
-                ZL_WAIT(&sm.kx_empty, (item_cnt & 1) ^ 1, 6);
-                if (rank == 0) mbar_arrive_expect_tx(&sm.kv_full, 2 * (2 * Smem::kTileBytes + 2 * Smem::kBoxBytes));
-                for (int b = 0; b < 2; ++b) {
-                    tma_load_3d_pair(sm.k + b * Smem::kBoxBytes, &tm_k, kv_full_l, b * 64, wi.head, key0 + 128 * (int)rank);
-                    tma_load_3d_pair(sm.v + b * Smem::kBoxBytes, &tm_v, kv_full_l, b * 64, wi.head, key0 + 128 * (int)rank);
-                    tma_load_3d_pair(sm.kx[b], &tm_k, kv_full_l, 64 * (int)rank, wi.head, key0 + 128 * b);
-                }
+                ZL_WAIT(&sm.k_empty, (item_cnt & 1) ^ 1, 1);
+                if (rank == 0) mbar_arrive_expect_tx(&sm.k_full, 2 * Smem::kTileBytes);
+                for (int b = 0; b < 2; ++b)
+                    tma_load_3d_pair(sm.k + b * Smem::kBoxBytes, &tm_k, k_full_l, b * 64, wi.head, key0 + 128 * (int)rank);
+                ZL_WAIT(&sm.v_empty, (item_cnt & 1) ^ 1, 6);
+                if (rank == 0) mbar_arrive_expect_tx(&sm.v_full, 2 * Smem::kTileBytes);
+                for (int b = 0; b < 2; ++b)
+                    tma_load_3d_pair(sm.v + b * Smem::kBoxBytes, &tm_v, v_full_l, b * 64, wi.head, key0 + 128 * (int)rank);
                 #pragma unroll 1
                 for (int ti = 0; ti < g.n_tasks; ++ti) {
                     const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
@@ -280,11 +286,18 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // Its buffer is released two MMAs later than the Q rows; a producer of its own keeps that wait
             // from delaying the other loads.
             const uint32_t qc_full_l = map_to_cta(smem_u32(&sm.qc_full), 0);
-            uint32_t it_cnt = 0;
+            const uint32_t kx_full_l = map_to_cta(smem_u32(&sm.kx_full), 0);
+            uint32_t item_cnt = 0, it_cnt = 0;
             #pragma unroll 1
-            for (int it = cluster_id; it < p.n_items; it += n_clusters) {
+            for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
+                // the K columns for dQ are the last buffer of the previous item to come free (after its last dQ), and
+                // dQ is the last MMA group of a tile to need its operand: loaded here, off the other producer's path
+                ZL_WAIT(&sm.kx_empty, (item_cnt & 1) ^ 1, 8);
+                if (rank == 0) mbar_arrive_expect_tx(&sm.kx_full, 2 * 2 * Smem::kBoxBytes);
+                for (int b = 0; b < 2; ++b)
+                    tma_load_3d_pair(sm.kx[b], &tm_k, kx_full_l, 64 * (int)rank, wi.head, g.kv_off + wi.row0 + 128 * b);
                 #pragma unroll 1
                 for (int ti = 0; ti < g.n_tasks; ++ti) {
                     const Task t = p.tasks[p.kv_group_tasks[g.task_begin + ti]];
@@ -365,11 +378,11 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const WorkItem wi = p.items[it];
                 const KvGroup g = p.kv_groups[wi.unit];
                 const int n_it = count_q_tiles(p, g);
-                ZL_WAIT_WARP_CL(&sm.kv_full, item_cnt & 1, 11);
                 // Order of this warp's MMAs: dK(i) dP(i+1) dV(i+1) S(i+2); dQ(i) comes from the second issuer.  The
                 // two steps before the item's first tile (i = -2, -1) are the prologue: S(0), then dP(0) dV(0) S(1).
                 // S^T(x) overwrites the columns of dQ(x-2) (dQ(x-1) is only issued once S^T(x) has been read); the
-                // first S^T of an item follows the previous item's last dQ.
+                // first S^T of an item follows the previous item's last dQ, which cannot wait for it: the P/dS warps
+                // read that S^T only after their epilogue, and the epilogue stages in the boxes the last dQ reads.
                 #pragma unroll 1
                 for (int i = -2; i < n_it; ++i) {
                     if (i >= 0) {
@@ -388,8 +401,10 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         // dP^T of the next tile right behind it (it overwrites dS^T: ordered after dK on the tensor pipe)
                         const uint32_t c = it_base + i + 1;
                         ZL_WAIT_WARP_CL(&sm.dor_full, c & 1, 19);
+                        if (i + 1 == 0) ZL_WAIT_WARP_CL(&sm.v_full, item_cnt & 1, 12);
                         tc_fence_after();
                         issue_dp();
+                        if (i + 1 == n_it - 1 && mma_lane) mma_commit_pair(&sm.v_empty);  // the item's last dP^T: V may go
                         ZL_WAIT_WARP_CL(&sm.p_full, c & 1, 21);
                         ZL_WAIT_WARP_CL(&sm.doc_full, c & 1, 29);
                         tc_fence_after();
@@ -399,14 +414,15 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         const uint32_t c = it_base + i + 2;
                         const uint32_t drained = it_base + (i + 1 > 0 ? i + 1 : 0);  // dQ tiles that must have left TMEM
                         ZL_WAIT_WARP_CL(&sm.qr_full, c & 1, 22);
+                        if (i + 2 == 0) ZL_WAIT_WARP_CL(&sm.k_full, item_cnt & 1, 11);
                         while (dq_waited < drained) { ZL_WAIT_WARP_CL(&sm.dq_empty[dq_waited & 1], (dq_waited >> 1) & 1, 25); ++dq_waited; }
                         tc_fence_after();
                         issue_s();  // overwrites P^T: ordered after dV on the tensor pipe
+                        if (i + 2 == n_it - 1 && mma_lane) mma_commit_pair(&sm.k_empty);  // the item's last S^T: K may go
                     }
                 }
                 it_base += n_it;
                 if (mma_lane) mma_commit_pair(&sm.acc_full);
-                if (mma_lane) mma_commit_pair(&sm.kv_empty);
             }
         } else if (warp == 3 && rank == 0) {
             // -------------------------------------------------------------- second MMA issuer (leader CTA): dQ
@@ -422,7 +438,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
                 const KvGroup g = p.kv_groups[p.items[it].unit];
                 const int n_it = count_q_tiles(p, g);
-                ZL_WAIT_WARP_CL(&sm.kv_full, item_cnt & 1, 51);  // the K columns of this item are in place
+                ZL_WAIT_WARP_CL(&sm.kx_full, item_cnt & 1, 51);  // the K columns of this item are in place
                 #pragma unroll 1
                 for (int i = 0; i < n_it; ++i, ++it_cnt) {
                     ZL_WAIT_WARP_CL(&sm.ds_full, it_cnt & 1, 52);
