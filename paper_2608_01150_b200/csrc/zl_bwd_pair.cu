@@ -136,13 +136,7 @@ __device__ __forceinline__ bool pair_wait_cluster(uint64_t* bar, uint32_t parity
         }                                                                                     \
     } while (0)
 
-__device__ __forceinline__ int count_q_tiles(const BwdParams& p, const KvGroup& g) {
-    int n = 0;
-    #pragma unroll 1
-    for (int ti = 0; ti < g.n_tasks; ++ti)
-        n += (p.tasks[p.kv_group_tasks[g.task_begin + ti]].q_len + kTileQ - 1) / kTileQ;
-    return n;
-}
+__device__ __forceinline__ int count_q_tiles(const BwdParams&, const KvGroup& g) { return g.n_q_tiles; }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_q64,
@@ -477,10 +471,16 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const float sl2 = p.scale_log2;
         uint32_t item_cnt = 0, it_cnt = 0;
         bool store_pending = false;  // warp-uniform
+        // The item after this one is fetched while this one runs: at an item boundary these warps are on the critical
+        // path (epilogue, then the next item's first P), and two dependent loads from global memory are ~1,200 cycles.
+        WorkItem wi_cur = p.items[min(cluster_id, p.n_items - 1)];
+        KvGroup g_cur = p.kv_groups[wi_cur.unit];
         #pragma unroll 1
         for (int it = cluster_id; it < p.n_items; it += n_clusters, ++item_cnt) {
-            const WorkItem wi = p.items[it];
-            const KvGroup g = p.kv_groups[wi.unit];
+            const WorkItem wi = wi_cur;
+            const KvGroup g = g_cur;
+            const bool has_next = it + n_clusters < p.n_items;
+            if (has_next) wi_cur = p.items[it + n_clusters];
             const int rows_here = min(kTileKV, wi.rows - kTileKV * (int)rank);  // key rows of this CTA's tile (may be <= 0)
             const bool row_ok = row < rows_here;
             const float row_bias = row_ok ? 0.f : -INFINITY;
@@ -583,6 +583,7 @@ zl_bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
             }
             // ---- epilogue: warpgroup 0 stores dV, warpgroup 1 stores dK (scaled), one key row per thread
+            if (has_next) g_cur = p.kv_groups[wi_cur.unit];  // arrives under the epilogue
             ZL_WAIT_WARP(&sm.acc_full, item_cnt & 1, 34);
             tc_fence_after();
             const float sc = (wg == 0) ? 1.f : p.scale;

@@ -46,6 +46,8 @@ struct alignas(32) QGroup {
 struct alignas(16) KvGroup {
     int32_t kv_off, kv_len;
     int32_t task_begin, n_tasks;  // range in the kv-group task list
+    int32_t n_q_tiles;            // 128-row query tiles of all its tasks together
+    int32_t pad_[3];
 };
 
 // One attention problem of a placement as the builder receives it: a whole sequence (q range ==

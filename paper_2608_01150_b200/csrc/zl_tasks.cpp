@@ -250,8 +250,11 @@ zl_status build_schedule(const std::vector<InputTask>& in, int32_t n_shards, int
         }
         for (size_t g = 0; g < kmembers.size(); ++g) {
             const Task& t0 = s->tasks[kmembers[g][0]];
-            KvGroup kgp{t0.kv_off, t0.kv_len, (int32_t)s->kv_group_tasks.size(), (int32_t)kmembers[g].size()};
-            for (int32_t ti : kmembers[g]) s->kv_group_tasks.push_back(ti);
+            KvGroup kgp{t0.kv_off, t0.kv_len, (int32_t)s->kv_group_tasks.size(), (int32_t)kmembers[g].size(), 0, {0, 0, 0}};
+            for (int32_t ti : kmembers[g]) {
+                s->kv_group_tasks.push_back(ti);
+                kgp.n_q_tiles += (s->tasks[ti].q_len + kTileQ - 1) / kTileQ;
+            }
             s->kv_groups.push_back(kgp);
         }
     }
