@@ -147,3 +147,44 @@ def test_sm_margin_changes_no_result():
         assert float((dQ.float() - dQ0.float()).norm() / dQ0.float().norm()) <= 1e-4
     with pytest.raises(run.Z.ZlError):
         run.h.set_sm_margin(-1)
+
+
+def test_phases_with_head_ranges():
+    """Whole images over all heads in phase 0; two Ulysses-shaped sequences over half of the heads each, sharing
+    one block of rows, released one after the other (the arrival of two all-to-all batches)."""
+    p = W.ulysses_mix_placement(n_heads=4, head_dim=128, n_images=3, image_len=700, seq_len=900, degree=2)
+    Q, K, V, dO = _inputs(p, 8)
+    ref = EngineRun(p)
+    O0, LSE0, _, _ = ref.forward(Q, K, V)
+    dQ0, dK0, dV0 = ref.backward(Q, K, V, O0, LSE0, dO)
+    run = EngineRun(p)
+    Z, h = run.Z, run.h
+    h.set_fwd_phases([0, 0, 0, 1, 2], None, 3)
+    h.set_bwd_phases([1, 1, 1, 0, 0], None, 2)
+    O, LSE, OP, LP = _buffers(p, h.info, Q.device)
+    # the Ulysses rows arrive head range by head range: fill them just before their phase
+    base = 3 * 700
+    Kt, Vt, Qt = K.clone(), V.clone(), Q.clone()
+    Kt[base:], Vt[base:], Qt[base:] = 0, 0, 0
+    Z.coalesced_attn_fwd_phase(h, 0, Qt, Kt, Vt, run.scale, O, LSE, OP, LP)
+    torch.cuda.synchronize()
+    for ph, (hb, he) in ((1, (0, 2)), (2, (2, 4))):
+        Qt[base:, hb:he], Kt[base:, hb:he], Vt[base:, hb:he] = Q[base:, hb:he], K[base:, hb:he], V[base:, hb:he]
+        Z.coalesced_attn_fwd_phase(h, ph, Qt, Kt, Vt, run.scale, O, LSE, OP, LP)
+        torch.cuda.synchronize()
+    Z.lse_merge(h, OP, LP, O, LSE)
+    torch.cuda.synchronize()
+    assert _same_bits(O, O0) and _same_bits(LSE, LSE0)
+    H, d = p.n_heads, p.head_dim
+    dQ = torch.full((p.total_q, H, d), SENTINEL, dtype=torch.bfloat16, device=Q.device)
+    dK, dV = torch.full_like(dQ, SENTINEL), torch.full_like(dQ, SENTINEL)
+    nbytes = int(h.info.bwd_workspace_bytes)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=Q.device)
+    Z.coalesced_attn_bwd_phase(h, 0, Q, K, V, O, LSE, dO, run.scale, dQ, dK, dV, ws, nbytes)
+    torch.cuda.synchronize()
+    assert _same_bits(dK[base:], dK0[base:]) and _same_bits(dV[base:], dV0[base:]) and bool((dK[:base] == SENTINEL).all())
+    Z.coalesced_attn_bwd_phase(h, 1, Q, K, V, O, LSE, dO, run.scale, dQ, dK, dV, ws, nbytes)
+    torch.cuda.synchronize()
+    assert h.last_device_status()[0] == 0
+    assert _same_bits(dK, dK0) and _same_bits(dV, dV0)
+    assert float((dQ.float() - dQ0.float()).norm() / dQ0.float().norm()) <= 1e-4

@@ -362,3 +362,49 @@ def test_a_fused_range_runs_in_the_latest_phase_of_its_chunks(Z):
     fi, _ = h.phase_info()
     assert fi[1] == 0 and fi[2] > 0 and fi[0] > 0
     assert all(t == 2 for (t, _, _, _) in h.fwd_items()[fi[0]:])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_phase_assignments_partition_both_lists(Z, seed):
+    """Whatever phases the caller asks for: every forward item sits in the phase of its task, every backward item in
+    the latest phase among the tasks of its kv group, nothing is lost or duplicated, and the order inside a phase is
+    the order the single-phase list had."""
+    rng = np.random.RandomState(100 + seed)
+    p = W.random_placement(rng, int(rng.randint(1, 4)), 64, max_whole=5, max_len=700, max_groups=3)
+    h = _build(Z, p)
+    tasks = _tasks_of(p)
+    f0, b0 = h.fwd_items(), h.bwd_items()
+    n_whole, n_shards = len(p.cu_seqlens) - 1, len(p.shards)
+    n_phases = int(rng.randint(1, 6))
+    wp = [int(x) for x in rng.randint(0, n_phases, n_whole)]
+    sp = [int(x) for x in rng.randint(0, n_phases, n_shards)]
+    h.set_fwd_phases(wp, sp, n_phases)
+    h.set_bwd_phases(wp, sp, n_phases)
+    # task numbering: whole sequences with len > 0, then shards with q_len > 0
+    task_phase = [wp[i] for i in range(n_whole) if p.cu_seqlens[i + 1] > p.cu_seqlens[i]] + \
+                 [sp[j] for j in range(n_shards) if p.shards[j][1] > 0]
+    assert len(task_phase) == len(tasks)
+    fi, bi = h.phase_info()
+    assert len(fi) == n_phases and len(bi) == n_phases
+    f1, b1 = h.fwd_items(), h.bwd_items()
+    assert sorted(f1) == sorted(f0) and sorted(b1) == sorted(b0)
+    pos = 0
+    for ph, n in enumerate(fi):
+        assert all(task_phase[t] == ph for (t, _, _, _) in f1[pos:pos + n])
+        assert f1[pos:pos + n] == [x for x in f0 if task_phase[x[0]] == ph]      # stable
+        pos += n
+    # kv groups in order of first appearance over the tasks with keys
+    group_of_range, group_phase = {}, []
+    for ti, t in enumerate(tasks):
+        if t[3] == 0:
+            continue
+        g = group_of_range.setdefault((t[2], t[3]), len(group_of_range))
+        if g == len(group_phase):
+            group_phase.append(task_phase[ti])
+        else:
+            group_phase[g] = max(group_phase[g], task_phase[ti])
+    pos = 0
+    for ph, n in enumerate(bi):
+        assert all(group_phase[g] == ph for (g, _, _, _) in b1[pos:pos + n])
+        assert b1[pos:pos + n] == [x for x in b0 if group_phase[x[0]] == ph]
+        pos += n
